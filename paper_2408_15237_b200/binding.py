@@ -14,10 +14,7 @@ from pathlib import Path
 
 import torch
 
-import os
-
-# MAMBA_SPEC_LIB points at another build of the same library (e.g. a debug build); default: the in-tree one.
-_LIB_PATH = Path(os.environ.get("MAMBA_SPEC_LIB") or Path(__file__).resolve().parent / "libmamba_spec.so")
+_LIB_PATH = Path(__file__).resolve().parent / "libmamba_spec.so"
 if not _LIB_PATH.exists():
     raise ImportError(
         f"{_LIB_PATH} is missing: build it with `python -m paper_2408_15237_b200.build` "

@@ -62,24 +62,16 @@ __device__ __forceinline__ int load_n_prev(const VerifyParams &p, int b) {
 // Launchers (defined in verify_generic.cu / verify_stream.cu).  Return cudaGetLastError().
 cudaError_t launch_verify_generic(const VerifyParams &p, bool bf16, cudaStream_t stream);
 
-// Launch-shape knobs of the streaming kernel; 0 (lead: -1) = let the planner choose.
-struct Tuning {
-    int stages = 0;       // depth of the state ring
-    int grid = 0;         // number of CTAs (default: one per SM)
-    int raw_stages = 0;   // depth of the ring of small-input stages
-    int lead = -1;        // chunks by which small-input copies run ahead of state copies
-};
-
 // Shared-memory plan of the streaming kernel: ring depths and byte offsets (all multiples of 16).
 struct StreamLayout {
-    int S, R;           // stages of the state ring and of the raw-input ring
-    int ngroups;        // compute groups in use (each needs a buffer)
-    int TCAP, JCAP;     // token rows / replayed tokens the buffers are sized for
-    int lead;           // chunks by which the small-input copies run ahead of the state copies
-    float inv_hpg_b, inv_hpg_c;   // 1 / (heads per B group), 1 / (heads per C group)
+    int S;              // stages of the state ring (one unit = 32 state rows each)
+    int AW;             // compute warps in use; S is a multiple of it
+    int TCAP, JB;       // token rows the tables are sized for; B rows kept as fp32
+    int hpg_b, hpg_c;   // heads per B group, heads per C group
+    unsigned H_mul, uph_mul;   // ceil(2^32 / H), ceil(2^32 / (P/32)): division by multiply-high
     int state_off, state_stride;
-    int raw_off, raw_stride, raw_tx, r_x, r_z, r_B, r_C, r_dt, r_cst, r_cw, r_cb;   // raw_tx: bytes one fill brings in
-    int grp_off, grp_stride, c_Cf, c_Bf, c_gz, c_xc, c_G, c_hc, c_part;   // per compute group
+    // a table slot (one per head warp): what a head warp derives from a head's dt, B and C rows
+    int tab_off, tab_stride, c_Cf, c_Bf, c_G, c_hc;
 };
 struct StreamPlan {
     bool ok;
@@ -88,8 +80,17 @@ struct StreamPlan {
     StreamLayout layout;
     char name[112];
 };
-StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, size_t smem_per_block_optin,
-                              const Tuning &tune);
-cudaError_t launch_verify_stream(const VerifyParams &p, const StreamPlan &plan, cudaStream_t stream);
+// Tensor maps of one launch (opaque 128-byte descriptors, the driver's CUtensorMap).
+struct alignas(64) TensorMapBytes {
+    unsigned char opaque[128];
+};
+struct alignas(64) InputMaps {
+    TensorMapBytes state;    // [32 columns][rows][N/32 quarters], 128-byte swizzle
+    TensorMapBytes state_k;  // the same over the second snapshot's buffer (FLAG_STATE_K only)
+};
+StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, size_t smem_per_block_optin);
+// Encodes the tensor maps of a launch (host work: driver calls); false if the driver refuses.
+bool encode_stream_maps(const VerifyParams &p, const StreamPlan &plan, InputMaps *tm);
+cudaError_t launch_verify_stream(const VerifyParams &p, const StreamPlan &plan, const InputMaps &tm, cudaStream_t stream);
 
 }  // namespace mspec
