@@ -38,6 +38,7 @@ constexpr int kFlagGate = 1;
 constexpr int kFlagConvSilu = 2;
 constexpr int kFlagYF32 = 4;
 constexpr int kFlagStateK = 8;
+constexpr int kFlagEarlyState = 16;   // in VerifyParams::flags only when the host has checked that it may be used
 constexpr int kStatusNprevClamped = 1;
 constexpr int kStatusAcceptClamped = 2;
 constexpr int kStatusCopyTimeout = 4;

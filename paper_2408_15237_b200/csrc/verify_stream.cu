@@ -464,9 +464,8 @@ struct RowIn {
     float bias;
 };
 template <int TC>
-__device__ __forceinline__ void load_row(const VerifyParams &p, int b, int h, int row, RowIn<TC> &in) {
-    const int HP = p.H * p.P;
-    const int tlim = p.t_max < TC ? p.t_max : TC;   // rows of the slab; those past the sequence's tokens are never used
+__device__ __forceinline__ void load_row(const VerifyParams &p, int b, int h, int row, int tlim, RowIn<TC> &in) {
+    const int HP = p.H * p.P;   // tlim: token rows to load (at most the rows of the slab)
     const unsigned short *xg = reinterpret_cast<const unsigned short *>(p.x) + ((size_t)b * p.t_max * p.H + h) * p.P + row;
     const unsigned short *zg = reinterpret_cast<const unsigned short *>(p.z) + ((size_t)b * p.t_max * p.H + h) * p.P + row;
     const unsigned short *cg = reinterpret_cast<const unsigned short *>(p.conv_state) + (size_t)b * (kW - 1) * HP + h * p.P + row;
@@ -478,6 +477,47 @@ __device__ __forceinline__ void load_row(const VerifyParams &p, int b, int h, in
     for (int t = 0; t < TC; ++t) in.zr[t] = (p.z != nullptr && t < tlim) ? zg[t * HP] : (unsigned short)0;
     in.wv = reinterpret_cast<const float4 *>(p.conv_w)[h * p.P + row];
     in.bias = p.conv_b[h * p.P + row];
+}
+
+// The same addresses as load_row / load_head, as L2 prefetches: they have no architectural effect, so they may go
+// out before the previous kernel of the stream has completed, and they take the cold misses (address translation,
+// first DRAM access) off the path of the real loads.
+__device__ __forceinline__ void prefetch_l2(const void *ptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr)); }
+template <int TC>
+__device__ __forceinline__ void prefetch_row(const VerifyParams &p, int b, int h, int row, int tlim) {
+    const int HP = p.H * p.P;
+    const unsigned short *xg = reinterpret_cast<const unsigned short *>(p.x) + ((size_t)b * p.t_max * p.H + h) * p.P + row;
+    const unsigned short *zg = reinterpret_cast<const unsigned short *>(p.z) + ((size_t)b * p.t_max * p.H + h) * p.P + row;
+    const unsigned short *cg = reinterpret_cast<const unsigned short *>(p.conv_state) + (size_t)b * (kW - 1) * HP + h * p.P + row;
+    if ((row & 15) == 0) {   // one lane per 32-byte sector
+#pragma unroll
+        for (int wi = 0; wi < kW - 1; ++wi) prefetch_l2(cg + wi * HP);
+#pragma unroll
+        for (int t = 0; t < TC; ++t) {
+            if (t < tlim) {
+                prefetch_l2(xg + t * HP);
+                if (p.z != nullptr) prefetch_l2(zg + t * HP);
+            }
+        }
+    }
+    if ((row & 1) == 0) prefetch_l2(reinterpret_cast<const float4 *>(p.conv_w) + h * p.P + row);
+    if ((row & 7) == 0) prefetch_l2(p.conv_b + h * p.P + row);
+}
+template <int N, int TC>
+__device__ __forceinline__ void prefetch_head(const VerifyParams &p, const StreamLayout &L, const Work &w, int head, int lane) {
+    const int b = div_H(w, head), h = head - b * w.H;
+    const size_t trow = (size_t)b * p.t_max;
+    const int rows = p.t_max < TC ? p.t_max : TC, r = lane >> 1;   // lane -> (row, half of a 256-byte row)
+    const __nv_bfloat16 *Cg = reinterpret_cast<const __nv_bfloat16 *>(p.C) + ((trow * p.GC) + h / L.hpg_c) * N;
+    const __nv_bfloat16 *Bg = reinterpret_cast<const __nv_bfloat16 *>(p.B) + ((trow * p.GB) + h / L.hpg_b) * N;
+    if (r < rows) {
+        if ((lane & 1) * 64 < N) {
+            prefetch_l2(Cg + (size_t)r * p.GC * N + (lane & 1) * 64);
+            prefetch_l2(Bg + (size_t)r * p.GB * N + (lane & 1) * 64);
+        }
+        if ((lane & 1) == 0) prefetch_l2(reinterpret_cast<const __nv_bfloat16 *>(p.dt) + (trow + r) * p.H + h);
+    }
+    if (lane == 0) { prefetch_l2(p.A + h); prefetch_l2(p.D + h); }
 }
 
 // The streaming part over one block of NT tokens.  The rows sit in the stage as the TMA engine wrote them:
@@ -509,8 +549,12 @@ __device__ __forceinline__ void stream_block(unsigned char *rb, uint32_t gx, con
             for (int i = 0; i < 4; ++i) acc[t][i] = ffma2(hi2(hv[i]), hi2(cv), acc[t][i]);
         }
         if (FORM) {
+            const float2 aj2 = make_float2(aj, aj);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) hv[i] = make_float4(hv[i].x * aj, hv[i].y * aj, hv[i].z * aj, hv[i].w * aj);
+            for (int i = 0; i < 4; ++i) {
+                const float2 l = __fmul2_rn(lo2(hv[i]), aj2), h2 = __fmul2_rn(hi2(hv[i]), aj2);
+                hv[i] = make_float4(l.x, l.y, h2.x, h2.y);
+            }
 #pragma unroll
             for (int s = 0; s < JC; s += 2) {
                 if (s < j) {   // two at a time: a coefficient past j is zero and its B row is zeros
@@ -521,7 +565,9 @@ __device__ __forceinline__ void stream_block(unsigned char *rb, uint32_t gx, con
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const float c = HOIST ? cfr[HOIST ? s + e : 0][i] : __shfl_sync(0xffffffffu, cx[s + e], g + 8 * i);
-                                hv[i] = make_float4(fmaf(c, bv.x, hv[i].x), fmaf(c, bv.y, hv[i].y), fmaf(c, bv.z, hv[i].z), fmaf(c, bv.w, hv[i].w));
+                                const float2 c2 = make_float2(c, c);
+                                const float2 l = ffma2(c2, lo2(bv), lo2(hv[i])), h2 = ffma2(c2, hi2(bv), hi2(hv[i]));
+                                hv[i] = make_float4(l.x, l.y, h2.x, h2.y);
                             }
                         }
                     }
@@ -553,10 +599,16 @@ __device__ __forceinline__ bool compute_unit(const VerifyParams &p, const Stream
     // ---- causal conv + SiLU of this row over the token block, from the rolling window
     float xc[TC];
 #pragma unroll
-    for (int t = 0; t < TC; ++t) {
-        const float v = fmaf(in.wv.w, bf16_bits_to_f32(in.xr[t + 3]), fmaf(in.wv.z, bf16_bits_to_f32(in.xr[t + 2]),
-                        fmaf(in.wv.y, bf16_bits_to_f32(in.xr[t + 1]), fmaf(in.wv.x, bf16_bits_to_f32(in.xr[t]), in.bias))));
-        xc[t] = conv_silu ? silu_fast(v) : v;
+    for (int t2 = 0; t2 < TC; t2 += 2) {
+        xc[t2] = xc[t2 + 1] = 0.f;
+        if (t2 < T) {   // tokens in pairs; a token past T gives a value that is never used
+#pragma unroll
+            for (int t = t2; t < t2 + 2; ++t) {
+                const float v = fmaf(in.wv.w, bf16_bits_to_f32(in.xr[t + 3]), fmaf(in.wv.z, bf16_bits_to_f32(in.xr[t + 2]),
+                                fmaf(in.wv.y, bf16_bits_to_f32(in.xr[t + 1]), fmaf(in.wv.x, bf16_bits_to_f32(in.xr[t]), in.bias))));
+                xc[t] = conv_silu ? silu_fast(v) : v;
+            }
+        }
     }
 
     // ---- the head's tables: published by the slot's head warp.  The counter tells which use of the slot is
@@ -576,6 +628,8 @@ __device__ __forceinline__ bool compute_unit(const VerifyParams &p, const Stream
         const float *Gm = reinterpret_cast<const float *>(slot + L.c_G);
 #pragma unroll
         for (int t = 0; t < TC; ++t) {
+            ya[t] = yw[t] = 0.f;
+            if ((t & ~1) >= T) continue;   // tokens in pairs, as above
             float wsum = 0.f;
 #pragma unroll
             for (int s4 = 0; s4 <= t; s4 += 4) {
@@ -756,15 +810,14 @@ __device__ __forceinline__ void compute_role(const VerifyParams &p, const Stream
     // Warp w takes units w, w + AW, ... through its own stages w, w + AW, ... (S / AW of them, in turn): every
     // use of a stage is requested and waited for by the same warp, in order, so a wait is never more than one
     // phase behind its barrier, and no "empty" barrier is needed.
-    const int spw = L.S / L.AW;
-    int k = 0;
+    int k = 0, ss = warp, sp = 0;
     for (int n = warp; n < w.nunits; n += L.AW, ++k) {
         int m, head, u;
         unit_of(w, n, m, head, u);
-        const int hs = m % kSlots, turn = k % spw, ss = warp + turn * L.AW, sp = (k / spw) & 1;
+        const int hs = m % kSlots;
         const int b = div_H(w, head), h = head - b * w.H;
-        if (k > 0) load_row<TC>(p, b, h, u * kUnitRows + lane, in);   // (the first unit's loads went out at the start of the kernel)
         const int j = pending_of(p, ctl, b), T = j + p.k;
+        if (k > 0) load_row<TC>(p, b, h, u * kUnitRows + lane, T, in);   // (the first unit's loads went out at the start of the kernel)
         const bool ok = compute_unit<N, TC, JC, SNAP>(p, L, tm, ctl, smem + L.state_off + (size_t)ss * L.state_stride,
                                                        smem + L.tab_off + (size_t)hs * L.tab_stride, smem_u32(&ctl.state_full[ss]),
                                                        (uint32_t)sp, hs, m, ss, n + L.S, smem, w, head, b, h, u, j, T, lane, in);
@@ -775,6 +828,8 @@ __device__ __forceinline__ void compute_role(const VerifyParams &p, const Stream
             }
             return;
         }
+        ss += L.AW;
+        if (ss >= L.S) { ss = warp; sp ^= 1; }
     }
 }
 
@@ -786,9 +841,6 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
     extern __shared__ __align__(1024) unsigned char smem[];
     Ctrl &ctl = *reinterpret_cast<Ctrl *>(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // Programmatic dependent launch: let the next kernel of the stream take SMs as this grid drains ...
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
     if (tid == 0) {
         make_work(p, L, *reinterpret_cast<Work *>(ctl.work));
         for (int s = 0; s < L.S; ++s) {
@@ -805,9 +857,33 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
     }
     __syncthreads();
     const Work &w = *reinterpret_cast<const Work *>(ctl.work);   // left in shared memory: read where needed
-    // Nothing else touches global memory before everything launched earlier in the stream has completed:
-    // only the set-up above overlaps with the previous kernel's tail.
+    // Programmatic dependent launch.  Nothing touches global memory before everything launched earlier in the
+    // stream has completed -- except, where the caller has promised that the kernel before this one does not
+    // write this call's state, the first state requests: the rows then stream in while the previous kernel's
+    // last CTAs finish.  The next kernel is let in only after the wait, so that its own early requests can
+    // overlap with this kernel but with nothing older.
+    const bool early = (p.flags & kFlagEarlyState) != 0;
+    auto first_requests = [&]() {
+        if (warp < L.AW && lane == 0)
+            for (int n = warp, ss = warp; n < w.nunits && ss < L.S; n += L.AW, ss += L.AW) request_state<N>(p, L, smem, ctl, tm, w, n, ss, 0);
+    };
+    if (early) first_requests();
+    {   // what every warp will load first, as prefetches
+        const int tl = p.t_max < TC ? p.t_max : TC;
+        if (tid < (p.batch < kJTable ? p.batch : kJTable)) prefetch_l2(p.n_prev + tid);
+        if (warp >= kComputeWarps) {
+            const int hw = warp - kComputeWarps;
+            if (hw < w.nitems) prefetch_head<N, TC>(p, L, w, item_of(w, hw).head, lane);
+            if (hw + kHeadWarps < w.nitems) prefetch_head<N, TC>(p, L, w, item_of(w, hw + kHeadWarps).head, lane);
+        } else if (warp < L.AW && warp < w.nunits) {
+            int m, head, u;
+            unit_of(w, warp, m, head, u);
+            const int b = div_H(w, head);
+            prefetch_row<TC>(p, b, head - b * w.H, u * kUnitRows + lane, tl);
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // Every warp sends its small loads first and the state requests behind them: behind the state requests of
     // 148 CTAs the small loads would wait for microseconds.
     const int ntab = p.batch < kJTable ? p.batch : kJTable;
@@ -825,9 +901,9 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
             int m, head, u;
             unit_of(w, warp, m, head, u);
             const int b = div_H(w, head);
-            load_row<TC>(p, b, head - b * w.H, u * kUnitRows + lane, in);
-            if (lane == 0)
-                for (int n = warp, ss = warp; n < w.nunits && ss < L.S; n += L.AW, ss += L.AW) request_state<N>(p, L, smem, ctl, tm, w, n, ss, 0);
+            // (the pending length is not known yet: all rows of the slab, those past the sequence's tokens are never used)
+            load_row<TC>(p, b, head - b * w.H, u * kUnitRows + lane, p.t_max < TC ? p.t_max : TC, in);
+            if (!early) first_requests();
         }
 #pragma unroll 1
         for (int i = tid; i < ntab; i += kThreads) ctl.jarr[i] = load_n_prev(p, i);
