@@ -70,11 +70,6 @@ extern "C" {
 #define MAMBA_SPEC_FLAG_GATE 1      /* y <- y * SiLU(z); io->z must then be non-null */
 #define MAMBA_SPEC_FLAG_CONV_SILU 2 /* SiLU after the conv (else identity)           */
 #define MAMBA_SPEC_FLAG_Y_F32 4     /* y is float32 whatever the act dtype is        */
-#define MAMBA_SPEC_FLAG_EARLY_STATE 16 /* a promise by the caller: the kernel that precedes a verify call in its stream
-                                         never writes that call's state (true of a decode loop that goes from layer to
-                                         layer).  The streaming kernel then requests its first state rows while that
-                                         kernel is still finishing.  A call right behind this context's own call on the
-                                         same state ignores the flag.                                                 */
 #define MAMBA_SPEC_FLAG_STATE_K 8   /* second snapshot: the cache after ALL T_b tokens, to io->state_k /
                                        io->conv_state_k (Algorithm 2 caches h_j and h_k; Fig. 2)  */
 

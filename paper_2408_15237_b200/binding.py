@@ -23,7 +23,7 @@ lib = ctypes.CDLL(str(_LIB_PATH))
 
 OK = 0
 DTYPE_F32, DTYPE_BF16 = 0, 1
-FLAG_GATE, FLAG_CONV_SILU, FLAG_Y_F32, FLAG_STATE_K, FLAG_EARLY_STATE = 1, 2, 4, 8, 16
+FLAG_GATE, FLAG_CONV_SILU, FLAG_Y_F32, FLAG_STATE_K = 1, 2, 4, 8
 STATUS_NPREV_CLAMPED, STATUS_ACCEPT_CLAMPED, STATUS_COPY_TIMEOUT = 1, 2, 4
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_STREAM = 0, 1, 2
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_MISALIGNED, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOT_INIT = -1, -2, -3, -4, -5, -6

@@ -38,7 +38,6 @@ constexpr int kFlagGate = 1;
 constexpr int kFlagConvSilu = 2;
 constexpr int kFlagYF32 = 4;
 constexpr int kFlagStateK = 8;
-constexpr int kFlagEarlyState = 16;   // in VerifyParams::flags only when the host has checked that it may be used
 constexpr int kStatusNprevClamped = 1;
 constexpr int kStatusAcceptClamped = 2;
 constexpr int kStatusCopyTimeout = 4;
@@ -65,14 +64,14 @@ cudaError_t launch_verify_generic(const VerifyParams &p, bool bf16, cudaStream_t
 
 // Shared-memory plan of the streaming kernel: ring depths and byte offsets (all multiples of 16).
 struct StreamLayout {
-    int S;              // stages of the state ring (one unit = 32 state rows each)
-    int AW;             // compute warps in use; S is a multiple of it
-    int TCAP, JB;       // token rows the tables are sized for; B rows kept as fp32
-    int hpg_b, hpg_c;   // heads per B group, heads per C group
-    unsigned H_mul, uph_mul;   // ceil(2^32 / H), ceil(2^32 / (P/32)): division by multiply-high
+    int S, R;           // stages of the state ring and of the raw-input ring
+    int ngroups;        // compute groups in use (each needs a buffer)
+    int TCAP, JCAP;     // token rows / replayed tokens the buffers are sized for
+    int lead;           // chunks by which the small-input copies run ahead of the state copies
+    float inv_hpg_b, inv_hpg_c;   // 1 / (heads per B group), 1 / (heads per C group)
     int state_off, state_stride;
-    // a table slot (one per head warp): what a head warp derives from a head's dt, B and C rows
-    int tab_off, tab_stride, c_Cf, c_Bf, c_G, c_hc;
+    int raw_off, raw_stride, raw_tx, r_x, r_z, r_B, r_C, r_dt, r_cst, r_cw, r_cb;   // raw_tx: bytes one fill brings in
+    int grp_off, grp_stride, c_Cf, c_Bf, c_gz, c_xc, c_G, c_hc, c_part;   // per compute group
 };
 struct StreamPlan {
     bool ok;
@@ -81,16 +80,18 @@ struct StreamPlan {
     StreamLayout layout;
     char name[112];
 };
-// Tensor maps of one launch (opaque 128-byte descriptors, the driver's CUtensorMap).
+// Tensor maps of one launch (opaque 128-byte descriptors, the driver's CUtensorMap): one TMA request then
+// fetches the rows of all tokens of a chunk (the rows of one token are H*P apart in memory).
 struct alignas(64) TensorMapBytes {
     unsigned char opaque[128];
 };
 struct alignas(64) InputMaps {
+    TensorMapBytes x, z, B, C, dt, cst;
     TensorMapBytes state;    // [32 columns][rows][N/32 quarters], 128-byte swizzle
     TensorMapBytes state_k;  // the same over the second snapshot's buffer (FLAG_STATE_K only)
 };
 StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, size_t smem_per_block_optin);
-// Encodes the tensor maps of a launch (host work: driver calls); false if the driver refuses.
+// Encodes the tensor maps of a launch (host work: eight driver calls); false if the driver refuses.
 bool encode_stream_maps(const VerifyParams &p, const StreamPlan &plan, InputMaps *tm);
 cudaError_t launch_verify_stream(const VerifyParams &p, const StreamPlan &plan, const InputMaps &tm, cudaStream_t stream);
 

@@ -40,7 +40,6 @@ struct mamba_spec_ctx {
     int32_t *st_n_prev = nullptr;
     bool staging_ready = false;
     cudaStream_t last_stream = nullptr;
-    const void *last_state = nullptr, *last_state_k = nullptr;   // what this context's last verify launch wrote
     int32_t last_k = -1;
     int64_t launches = 0;
     std::vector<MapEntry> map_cache;   // empty for contexts that must not allocate
@@ -136,7 +135,7 @@ int mamba_spec_init(const mamba_spec_config *cfg, mamba_spec_ctx **out) {
     if (c.k_max < 0 || c.k_max > 32) return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: k_max %d outside 0..32", c.k_max);
     if (c.act_dtype != MAMBA_SPEC_DTYPE_F32 && c.act_dtype != MAMBA_SPEC_DTYPE_BF16)
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: unknown act_dtype %d", c.act_dtype);
-    if (c.flags & ~(MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K | MAMBA_SPEC_FLAG_EARLY_STATE))
+    if (c.flags & ~(MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K))
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: unknown flag bits 0x%x", c.flags);
     if (c.kernel_select < 0 || c.kernel_select > MAMBA_SPEC_KERNEL_STREAM)
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: unknown kernel_select %d", c.kernel_select);
@@ -221,16 +220,8 @@ static int check_and_fill(mamba_spec_ctx *ctx, VerifyParams &p, void *state, voi
     return MAMBA_SPEC_OK;
 }
 
-static int launch(mamba_spec_ctx *ctx, const VerifyParams &p_in, cudaStream_t stream, const char *who) {
+static int launch(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
     const mamba_spec_config &c = ctx->cfg;
-    VerifyParams p = p_in;
-    // Early state requests only where the promise can hold: never right behind this context's own launch on
-    // the same cache (or on a second snapshot that is now the cache).
-    p.flags &= ~kFlagEarlyState;
-    if ((c.flags & MAMBA_SPEC_FLAG_EARLY_STATE) && ctx->last_state != p.state && ctx->last_state_k != p.state)
-        p.flags |= kFlagEarlyState;
-    ctx->last_state = p.state;
-    ctx->last_state_k = p.state_k;
     const bool bf16 = c.act_dtype == MAMBA_SPEC_DTYPE_BF16;
     cudaError_t e;
     if (c.kernel_select == MAMBA_SPEC_KERNEL_AUTO || c.kernel_select == MAMBA_SPEC_KERNEL_STREAM) {
@@ -375,7 +366,7 @@ static int verify_host_static_impl(mamba_spec_ctx *tmp, void *state, void *conv_
         c.conv_width < 1 || c.conv_width > kMaxConvWidth || c.n_groups_b < 1 || c.n_groups_c < 1 ||
         c.n_heads % c.n_groups_b || c.n_heads % c.n_groups_c || c.k_max < 0 || c.k_max > 32 ||
         (c.act_dtype != MAMBA_SPEC_DTYPE_F32 && c.act_dtype != MAMBA_SPEC_DTYPE_BF16) ||
-        (c.flags & ~(MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K | MAMBA_SPEC_FLAG_EARLY_STATE)) || c.kernel_select < 0 ||
+        (c.flags & ~(MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K)) || c.kernel_select < 0 ||
         c.kernel_select > MAMBA_SPEC_KERNEL_STREAM || ((size_t)c.n_heads * c.head_dim * act_bytes(c)) % 16)
         return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: configuration rejected (same rules as mamba_spec_init)");
     if (!io) return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: io is null");
