@@ -58,6 +58,10 @@ def _lib():
         lib.oracle_step.argtypes = [ctypes.POINTER(_Dims)] + [dp] * 12 + [ip]
         lib.oracle_sequential.restype = ctypes.c_int
         lib.oracle_sequential.argtypes = [ctypes.POINTER(_Dims), ctypes.c_int32, ip] + [dp] * 12 + [ctypes.c_int32]
+        lib.oracle_verify_m1.restype = ctypes.c_int
+        lib.oracle_verify_m1.argtypes = [ctypes.POINTER(_Dims), ctypes.c_int32, ip] + [dp] * 14 + [ctypes.c_int32]
+        lib.oracle_step_m1.restype = ctypes.c_int
+        lib.oracle_step_m1.argtypes = [ctypes.POINTER(_Dims)] + [dp] * 12
         _LIB = lib
     return _LIB
 
@@ -168,3 +172,57 @@ def sequential(state, conv_state, x, dt, Bm, Cm, A, D, conv_w, conv_b, z, length
     if rc != 0:
         raise ValueError("oracle_sequential: lengths out of range")
     return y, state, conv_state
+
+
+def softplus_dt(dt_raw, bias):
+    """The sampling interval from its raw value: ``softplus(dt_raw + bias)`` with the bias broadcast over the
+    last axis (Sec. 2.2: the intervals come out of a network; a softplus keeps them positive)."""
+    v = np.asarray(dt_raw, dtype=np.float64) + np.asarray(bias, dtype=np.float64)
+    return np.where(v > 30.0, v, np.log1p(np.exp(np.minimum(v, 30.0))))
+
+
+def verify_m1(state, conv_state, x, dt, Bm, Cm, A, D, conv_w, conv_b, z, n_prev, k, flags, threads=1):
+    """Multi-step verification in the Mamba-1 parameterisation (Algorithm 1; Sec. 2.2): ``dt`` is
+    ``[Bt, Tmax, H*P]``, ``A`` is ``[H*P, N]``, ``D`` is ``[H*P]``.  Returns ``(y, state_out, conv_state_out)``."""
+    state, conv_state = _f64(state), _f64(conv_state)
+    Bt, H, P, N = state.shape
+    if N > 1024 or conv_state.shape[1] > 16:
+        raise ValueError("oracle_verify_m1 keeps a row of at most 1024 columns and 16 window slots on the stack")
+    x = _f64(x)
+    Tmax = x.shape[1]
+    Bm, Cm = _f64(Bm), _f64(Cm)
+    d = _dims(state, conv_state, Bm, Cm, Tmax, flags)
+    x = _f64(x, (Bt, Tmax, H, P))
+    dt = _f64(dt, (Bt, Tmax, H * P))
+    Bm, Cm = _f64(Bm, (Bt, Tmax, d.GB, N)), _f64(Cm, (Bt, Tmax, d.GC, N))
+    A, D = _f64(A, (H * P, N)), _f64(D, (H * P,))
+    conv_w, conv_b = _f64(conv_w, (H * P, d.W)), _f64(conv_b, (H * P,))
+    z = None if z is None else _f64(z, (Bt, Tmax, H, P))
+    n_prev = np.ascontiguousarray(np.asarray(n_prev, dtype=np.int32))
+    if n_prev.shape != (Bt,):
+        raise ValueError("n_prev shape")
+    y = np.full((Bt, Tmax, H, P), np.nan, dtype=np.float64)
+    s_out, c_out = np.empty_like(state), np.empty_like(conv_state)
+    rc = _lib().oracle_verify_m1(ctypes.byref(d), int(k), _ip(n_prev), _dp(state), _dp(conv_state), _dp(x), _dp(dt),
+                                 _dp(Bm), _dp(Cm), _dp(A), _dp(D), _dp(conv_w), _dp(conv_b), _dp(z),
+                                 _dp(y), _dp(s_out), _dp(c_out), int(threads))
+    if rc != 0:
+        raise ValueError("oracle_verify_m1: n_prev out of range for Tmax")
+    return y, s_out, c_out
+
+
+def step_m1(state, conv_state, x1, dt1, B1, C1, A, D, conv_w, conv_b, z1, flags):
+    """One decoding step of every sequence in the Mamba-1 parameterisation; returns ``(y1, state, conv_state)``."""
+    state, conv_state = _f64(state).copy(), _f64(conv_state).copy()
+    Bt, H, P, N = state.shape
+    B1, C1 = _f64(B1), _f64(C1)
+    d = _dims(state, conv_state, B1, C1, 1, flags)
+    x1, dt1 = _f64(x1, (Bt, H, P)), _f64(dt1, (Bt, H * P))
+    B1, C1 = _f64(B1, (Bt, d.GB, N)), _f64(C1, (Bt, d.GC, N))
+    A, D = _f64(A, (H * P, N)), _f64(D, (H * P,))
+    conv_w, conv_b = _f64(conv_w, (H * P, d.W)), _f64(conv_b, (H * P,))
+    z1 = None if z1 is None else _f64(z1, (Bt, H, P))
+    y1 = np.full((Bt, H, P), np.nan, dtype=np.float64)
+    _lib().oracle_step_m1(ctypes.byref(d), _dp(state), _dp(conv_state), _dp(x1), _dp(dt1), _dp(B1), _dp(C1),
+                          _dp(A), _dp(D), _dp(conv_w), _dp(conv_b), _dp(z1), _dp(y1))
+    return y1, state, conv_state

@@ -32,6 +32,13 @@
  * W-1 multiplies the current token, SiLU follows when enabled; the skip term
  * is D_h times the POST-conv x; the optional gate multiplies y by SiLU(z).
  *
+ * A second parameterisation, "Mamba-1" (Algorithm 1, Sec. 2.2: a sampling interval
+ * per channel and a dynamic A per (channel, state column), which is the form of
+ * the pure-Mamba verifiers of Table 1), has its own functions at the end of the
+ * file: oracle_verify_m1 / oracle_step_m1.  Reading taken there: the "N'" axis of
+ * Algorithm 1 is the channel axis of a head (P here), so dt is [.. H*P], A is
+ * [H*P][N] and the skip weight D is per channel.
+ *
  * Pins: multi-step == repeated oracle_step; multi-round accept/replay ==
  * oracle_sequential; dt=0, B=0, A->0 closed forms; causal linear attention as
  * a matmul; explicit unrolled sums on tiny inputs; numpy full convolution.
@@ -234,5 +241,119 @@ int oracle_sequential(const oracle_dims *d, int32_t L, const int32_t *len,
                         A, D, conv_w, conv_b, z ? z + bt * C : NULL, y + bt * C, NULL);
         }
     }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Mamba-1 parameterisation [Algorithm 1, Sec. 2.2]: the sampling interval is per channel and the
+ * dynamic A per (channel, state column):
+ *     h_t[p][n] = exp(dt_t[c] * A[c][n]) * h_{t-1}[p][n] + dt_t[c] * xc_t[p] * B_t[n],   c = h*P + p
+ *     y_t[p]    = sum_n C_t[n] * h_t[p][n] + D[c] * xc_t[p]        ( * SiLU(z_t[p]) when gated )
+ * Everything else (conv, groups, snapshot at the verified position) is as in oracle_verify.
+ * Layouts that differ:  dt [Bt][Tmax][H*P]   A [H*P][N]   D [H*P]
+ */
+int oracle_verify_m1(const oracle_dims *d, int32_t k, const int32_t *n_prev,
+                     const double *state, const double *conv_state,
+                     const double *x, const double *dt, const double *Bm, const double *Cm,
+                     const double *A, const double *D,
+                     const double *conv_w, const double *conv_b, const double *z,
+                     double *y, double *state_out, double *conv_state_out, int32_t nthreads)
+{
+    const int Bt = d->Bt, Tmax = d->Tmax, H = d->H, P = d->P, N = d->N, W = d->W;
+    const int C = H * P;
+    for (int b = 0; b < Bt; ++b)
+        if (n_prev[b] < 0 || n_prev[b] + k > Tmax) return -1;
+    if (nthreads < 1) nthreads = 1;
+
+#pragma omp parallel for collapse(2) num_threads(nthreads) schedule(dynamic, 1)
+    for (int b = 0; b < Bt; ++b) {
+        for (int c = 0; c < C; ++c) { /* every channel is its own recurrence */
+            const int h = c / P, j = n_prev[b], T = j + k;
+            const int gB = h / (H / d->GB), gC = h / (H / d->GC);
+            double hrow[1024]; /* N <= 1024 checked by the caller */
+            double win[16];
+            const double *st_in = state + ((size_t)b * C + c) * N;
+            double *st_out = state_out + ((size_t)b * C + c) * N;
+            for (int n = 0; n < N; ++n) hrow[n] = st_in[n];
+            for (int w = 0; w < W - 1; ++w) win[w] = conv_state[((size_t)b * (W - 1) + w) * C + c];
+            if (j == 0) {
+                for (int n = 0; n < N; ++n) st_out[n] = hrow[n];
+                for (int w = 0; w < W - 1; ++w) conv_state_out[((size_t)b * (W - 1) + w) * C + c] = win[w];
+            }
+            for (int t = 0; t < T; ++t) {
+                const size_t bt = (size_t)b * Tmax + t;
+                const double xin = x[bt * C + c];
+                double u = conv_b[c] + conv_w[c * W + (W - 1)] * xin;
+                for (int w = 0; w < W - 1; ++w) u += conv_w[c * W + w] * win[w];
+                if (d->flags & ORACLE_FLAG_CONV_SILU) u = silu(u);
+                for (int w = 0; w + 1 < W - 1; ++w) win[w] = win[w + 1];
+                if (W > 1) win[W - 2] = xin;
+                const double delta = dt[bt * C + c];
+                const double *Brow = Bm + (bt * d->GB + gB) * N, *Crow = Cm + (bt * d->GC + gC) * N;
+                double out = 0.0;
+                for (int n = 0; n < N; ++n) {
+                    hrow[n] = exp(delta * A[(size_t)c * N + n]) * hrow[n] + delta * u * Brow[n];
+                    out += Crow[n] * hrow[n];
+                }
+                out += D[c] * u;
+                if ((d->flags & ORACLE_FLAG_GATE) && z) out *= silu(z[bt * C + c]);
+                y[bt * C + c] = out;
+                if (t == j - 1) {
+                    for (int n = 0; n < N; ++n) st_out[n] = hrow[n];
+                    for (int w = 0; w < W - 1; ++w) conv_state_out[((size_t)b * (W - 1) + w) * C + c] = win[w];
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+/*
+ * One decoding step in the Mamba-1 parameterisation, written on its own: the whole batch goes through
+ * the conv first, then through the decay, then through the input term, then through the read-out, each
+ * as a separate sweep (another order of the same arithmetic than oracle_verify_m1's).  In place.
+ *   x1,z1,y1,dt1 : [Bt][H*P]   B1 : [Bt][GB][N]   C1 : [Bt][GC][N]
+ */
+int oracle_step_m1(const oracle_dims *d, double *state, double *conv_state,
+                   const double *x1, const double *dt1, const double *B1, const double *C1,
+                   const double *A, const double *D, const double *conv_w, const double *conv_b,
+                   const double *z1, double *y1)
+{
+    const int Bt = d->Bt, H = d->H, P = d->P, N = d->N, W = d->W, C = H * P;
+    double *u = (double *)malloc(sizeof(double) * (size_t)Bt * C);
+    for (int b = 0; b < Bt; ++b)
+        for (int c = 0; c < C; ++c) {
+            double s = conv_b[c];
+            for (int w = 0; w < W; ++w)
+                s += conv_w[c * W + w] * (w < W - 1 ? conv_state[((size_t)b * (W - 1) + w) * C + c] : x1[(size_t)b * C + c]);
+            u[(size_t)b * C + c] = (d->flags & ORACLE_FLAG_CONV_SILU) ? s / (1.0 + exp(-s)) : s;
+        }
+    for (int b = 0; b < Bt; ++b) {
+        double *cs = conv_state + (size_t)b * (W - 1) * C;
+        for (int w = 0; w < W - 2; ++w) memcpy(cs + (size_t)w * C, cs + (size_t)(w + 1) * C, sizeof(double) * C);
+        if (W > 1) memcpy(cs + (size_t)(W - 2) * C, x1 + (size_t)b * C, sizeof(double) * C);
+    }
+    for (int b = 0; b < Bt; ++b)        /* decay */
+        for (int c = 0; c < C; ++c)
+            for (int n = 0; n < N; ++n)
+                state[((size_t)b * C + c) * N + n] *= exp(A[(size_t)c * N + n] * dt1[(size_t)b * C + c]);
+    for (int b = 0; b < Bt; ++b)        /* input term */
+        for (int c = 0; c < C; ++c) {
+            const double *Bv = B1 + ((size_t)b * d->GB + (c / P) / (H / d->GB)) * N;
+            const double scale = dt1[(size_t)b * C + c] * u[(size_t)b * C + c];
+            for (int n = 0; n < N; ++n) state[((size_t)b * C + c) * N + n] += Bv[n] * scale;
+        }
+    for (int b = 0; b < Bt; ++b)        /* read-out */
+        for (int c = 0; c < C; ++c) {
+            const double *Cv = C1 + ((size_t)b * d->GC + (c / P) / (H / d->GC)) * N;
+            double out = D[c] * u[(size_t)b * C + c];
+            for (int n = 0; n < N; ++n) out += Cv[n] * state[((size_t)b * C + c) * N + n];
+            if ((d->flags & ORACLE_FLAG_GATE) && z1) {
+                const double g = z1[(size_t)b * C + c];
+                out *= g / (1.0 + exp(-g));
+            }
+            y1[(size_t)b * C + c] = out;
+        }
+    free(u);
     return 0;
 }

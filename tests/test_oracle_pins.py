@@ -308,3 +308,137 @@ def test_padding_rows_are_never_read():
     y, s_out, _ = oracle.verify(st, cv, b["x"], b["dt"], b["B"], b["C"], A, D, cw, cb, b["z"], b["n_prev"], s.k,
                                 s.flags)
     assert not np.isnan(s_out).any() and not np.isnan(y[0, :3]).any() and np.isnan(y[0, 3:]).all()
+
+
+# --------------------------------------------------------------------------- Mamba-1 parameterisation (Algorithm 1)
+def m1_problem(seed, **kw):
+    """small_problem with a sampling interval per channel, A per (channel, column) and D per channel."""
+    q = small_problem(seed, **kw)
+    g = np.random.default_rng(seed + 1000)
+    Bt, T, H, P = q["x"].shape
+    N = q["state"].shape[-1]
+    q["dt"] = np.log1p(np.exp(g.standard_normal((Bt, T, H * P)) - 1.0))
+    q["A"] = -np.exp(g.uniform(0, np.log(16), (H * P, N)))
+    q["D"] = g.standard_normal(H * P)
+    return q
+
+
+def run_verify_m1(q, n_prev, k, flags, **over):
+    a = dict(q, **over)
+    return oracle.verify_m1(a["state"], a["conv"], a["x"], a["dt"], a["B"], a["C"], a["A"], a["D"],
+                            a["cw"], a["cb"], a["z"], n_prev, k, flags)
+
+
+@pytest.mark.parametrize("flags", [0, GATE | CSILU])
+def test_m1_reduces_to_the_per_head_form_when_dt_and_A_are_constant_over_a_head(flags):
+    """Algorithm 1 with one interval and one A per head is the form the rest of this file pins."""
+    q = small_problem(21)
+    Bt, T, H, P = q["x"].shape
+    N = q["state"].shape[-1]
+    n_prev = np.array([0, 2, 3], dtype=np.int32)
+    y0, s0, c0 = run_verify(q, n_prev, 4, flags)
+    y1, s1, c1 = run_verify_m1(q, n_prev, 4, flags, dt=np.repeat(q["dt"], P, axis=2),
+                               A=np.repeat(q["A"], P)[:, None] * np.ones((1, N)), D=np.repeat(q["D"], P))
+    valid = ~np.isnan(y0)
+    assert (np.isnan(y1) == np.isnan(y0)).all()
+    np.testing.assert_allclose(y1[valid], y0[valid], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(s1, s0, rtol=1e-12, atol=1e-13)
+    np.testing.assert_array_equal(c1, c0)
+
+
+@pytest.mark.parametrize("flags", [0, GATE, CSILU, GATE | CSILU])
+def test_m1_multistep_equals_repeated_single_steps(flags):
+    q = m1_problem(22)
+    Bt, T, H, P = q["x"].shape
+    n_prev = np.zeros(Bt, dtype=np.int32)
+    y, _, _ = run_verify_m1(q, n_prev, T, flags)
+    st, cv = q["state"].copy(), q["conv"].copy()
+    for t in range(T):
+        y1, st, cv = oracle.step_m1(st, cv, q["x"][:, t], q["dt"][:, t], q["B"][:, t], q["C"][:, t], q["A"], q["D"],
+                                    q["cw"], q["cb"], q["z"][:, t], flags)
+        np.testing.assert_allclose(y[:, t], y1, rtol=1e-11, atol=1e-12)
+    # the snapshot after all tokens is what the single steps arrive at
+    _, s_all, c_all = run_verify_m1(q, np.full(Bt, T, dtype=np.int32), 0, flags)
+    np.testing.assert_allclose(s_all, st, rtol=1e-11, atol=1e-12)
+    np.testing.assert_array_equal(c_all, cv)
+
+
+def test_m1_unrolled_sums_by_brute_force():
+    """y_t[p] = sum_n C_t[n] ( exp(A[c,n] S_{0,t}) h0[p,n] + sum_{s<=t} exp(A[c,n] S_{s,t}) dt_s[c] xc_s[p] B_s[n] ) + D[c] xc_t[p],
+    S_{s,t} = sum_{s<r<=t} dt_r[c], written as explicit sums with no recurrence."""
+    q = m1_problem(23, Bt=2, H=2, P=3, N=4, GB=1, GC=2, T=5)
+    Bt, T, H, P = q["x"].shape
+    N = q["state"].shape[-1]
+    y, s_out, _ = run_verify_m1(q, np.array([2, 5], dtype=np.int32), 0, 0)
+    ylong, _, _ = run_verify_m1(q, np.zeros(Bt, dtype=np.int32), T, 0)
+    for b in range(Bt):
+        xc = full_conv_channels(q, b, 0)
+        for c in range(H * P):
+            h, p = divmod(c, P)
+            gB, gC = h // (H // 1), h // (H // 2)
+            for t in range(T):
+                tot = q["D"][c] * xc[t, c]
+                for n in range(N):
+                    acc = np.exp(q["A"][c, n] * q["dt"][b, :t + 1, c].sum()) * q["state"][b, h, p, n]
+                    for s in range(t + 1):
+                        acc += np.exp(q["A"][c, n] * q["dt"][b, s + 1:t + 1, c].sum()) * q["dt"][b, s, c] * xc[s, c] * q["B"][b, s, gB, n]
+                    tot += q["C"][b, t, gC, n] * acc
+                    if t + 1 == (2, 5)[b]:
+                        np.testing.assert_allclose(s_out[b, h, p, n], acc, rtol=1e-11, atol=1e-13)
+                np.testing.assert_allclose(ylong[b, t, h, p], tot, rtol=1e-11, atol=1e-13)
+
+
+def test_m1_closed_forms():
+    q = m1_problem(24)
+    Bt, T, H, P = q["x"].shape
+    N = q["state"].shape[-1]
+    full = np.full(Bt, T, dtype=np.int32)
+    # dt = 0: nothing moves, y = C . h0 + D xc
+    y, s, _ = run_verify_m1(q, full, 0, 0, dt=np.zeros_like(q["dt"]))
+    np.testing.assert_array_equal(s, q["state"])
+    for b in range(Bt):
+        xc = full_conv_channels(q, b, 0).reshape(T, H, P)
+        for h in range(H):
+            want = np.einsum("tn,pn->tp", q["C"][b, :, h // (H // 4)], q["state"][b, h]) + q["D"].reshape(H, P)[h] * xc[:, h]
+            np.testing.assert_allclose(y[b, :, h], want, rtol=1e-12, atol=1e-13)
+    # B = 0, constant interval per channel: every element decays by exp(A[c,n] T dt[c])
+    dtc = np.broadcast_to(q["dt"][:, :1], q["dt"].shape).copy()
+    _, s, _ = run_verify_m1(q, full, 0, 0, dt=dtc, B=np.zeros_like(q["B"]))
+    want = q["state"] * np.exp(q["A"].reshape(1, H, P, N) * (T * dtc[:, 0].reshape(Bt, H, P, 1)))
+    np.testing.assert_allclose(s, want, rtol=1e-12, atol=1e-14)
+    # A -> 0: a cumulative sum of rank-one terms dt_t[c] xc_t[p] B_t[n]
+    _, s, _ = run_verify_m1(q, full, 0, 0, A=np.zeros_like(q["A"]))
+    for b in range(Bt):
+        xc = full_conv_channels(q, b, 0).reshape(T, H, P)
+        for h in range(H):
+            upd = np.einsum("tp,tn->pn", q["dt"][b].reshape(T, H, P)[:, h] * xc[:, h], q["B"][b, :, h // (H // 2)])
+            np.testing.assert_allclose(s[b, h], q["state"][b, h] + upd, rtol=1e-12, atol=1e-13)
+
+
+def test_m1_snapshot_positions_and_untouched_rows():
+    q = m1_problem(25)
+    Bt, T, H, P = q["x"].shape
+    n_prev = np.array([0, 1, 3], dtype=np.int32)
+    y, s, c = run_verify_m1(q, n_prev, 3, GATE | CSILU)
+    for b in range(Bt):
+        assert np.isnan(y[b, n_prev[b] + 3:]).all() and not np.isnan(y[b, :n_prev[b] + 3]).any()
+        _, sb, cb = run_verify_m1(q, np.full(Bt, n_prev[b], dtype=np.int32), 0, GATE | CSILU)
+        np.testing.assert_allclose(s[b], sb[b], rtol=1e-12, atol=1e-14)
+        np.testing.assert_array_equal(c[b], cb[b])
+    np.testing.assert_array_equal(s[0], q["state"][0])
+
+
+# --------------------------------------------------------------------------- softplus of the raw interval
+def test_softplus_dt_against_its_identities():
+    g = np.random.default_rng(31)
+    v = g.uniform(-20, 20, (4, 5, 6))
+    bias = g.standard_normal(6)
+    sp = oracle.softplus_dt(v, bias)
+    u = v + bias
+    np.testing.assert_allclose(sp - oracle.softplus_dt(-v, -bias), u, rtol=1e-12, atol=1e-12)      # sp(u) - sp(-u) = u
+    np.testing.assert_allclose(np.expm1(sp), np.exp(u), rtol=1e-10)                                 # exp(sp(u)) = 1 + exp(u)
+    np.testing.assert_allclose(oracle.softplus_dt(np.zeros(3), np.zeros(3)), np.log(2.0))
+    eps = 1e-6                                                                                      # d sp / du = sigmoid
+    np.testing.assert_allclose((oracle.softplus_dt(v + eps, bias) - oracle.softplus_dt(v - eps, bias)) / (2 * eps),
+                               1.0 / (1.0 + np.exp(-u)), rtol=1e-6, atol=1e-9)
+    assert oracle.softplus_dt(np.array([100.0]), np.array([0.0]))[0] == 100.0
