@@ -72,6 +72,21 @@ extern "C" {
 #define MAMBA_SPEC_FLAG_Y_F32 4     /* y is float32 whatever the act dtype is        */
 #define MAMBA_SPEC_FLAG_STATE_K 8   /* second snapshot: the cache after ALL T_b tokens, to io->state_k /
                                        io->conv_state_k (Algorithm 2 caches h_j and h_k; Fig. 2)  */
+#define MAMBA_SPEC_FLAG_MAMBA1 16   /* Mamba-1 parameterisation (Algorithm 1, Sec. 2.2: the form of the paper's pure-Mamba
+                                       verifiers): the interval is per channel and A per channel and state column,
+                                         h_t[p,n] = exp(dt_t[c] * A[c][n]) * h_{t-1}[p,n] + dt_t[c] * xc_t[p] * B_t[n],
+                                         y_t[p]   = sum_n C_t[n] * h_t[p,n] + D[c] * xc_t[p],        c = h*P + p
+                                       with dt [batch][t_max][H*P], A [H*P][N], D [H*P].  Runs in the generic kernel. */
+#define MAMBA_SPEC_FLAG_DT_SOFTPLUS 32 /* dt arrives raw: the kernel uses softplus(dt + io->dt_bias) (Sec. 2.2: the
+                                       intervals come out of a network)                                            */
+#define MAMBA_SPEC_FLAG_COMMIT_SELECTS 64 /* needs FLAG_STATE_K.  Algorithm 2 keeps h_k when every draft was accepted and
+                                       h_j otherwise: (state, conv_state) and (io->state_k, io->conv_state_k) become two
+                                       equal buffers per sequence, one of which holds the sequence's cache.  A verify
+                                       call reads the cache where it is, puts the state at the verified position back
+                                       there and the state after all T_b tokens into the other buffer;
+                                       mamba_spec_commit then makes the other buffer the cache of every sequence with
+                                       accept_len == k_draft (nothing is pending for it any more) and records accept_len
+                                       as pending for the rest.  mamba_spec_get_selection tells where each cache is.   */
 
 /* bits of the device status word reported by mamba_spec_status */
 #define MAMBA_SPEC_STATUS_NPREV_CLAMPED 1  /* some n_prev_accepted[b] was outside [0, min(k_max, t_max-k)] */
@@ -115,6 +130,7 @@ typedef struct {
                             must not overlap state                                                  */
     void *conv_state_k;  /* DEVICE [batch][W-1][H*P] act dtype, output, FLAG_STATE_K only: the conv window
                             after all T_b tokens; must not overlap conv_state                       */
+    const float *dt_bias; /* DEVICE [H] float32 ([H*P] with FLAG_MAMBA1), FLAG_DT_SOFTPLUS only; null = no bias */
 } mamba_spec_io;
 
 /* HOST cfg, HOST out.  Validates the configuration, selects the device and
@@ -125,10 +141,12 @@ int mamba_spec_init(const mamba_spec_config *cfg, mamba_spec_ctx **out);
  *   state           [batch][H][P][N] float32, in/out: h_i -> h_{i+j_b}
  *   conv_state      [batch][W-1][H*P] act dtype, in/out, oldest row first
  *   x               [batch][t_max][H][P] act dtype, pre-conv inputs
- *   dt              [batch][t_max][H]    act dtype, already positive (post-softplus)
+ *   dt              [batch][t_max][H]    act dtype, already positive (post-softplus) unless FLAG_DT_SOFTPLUS;
+ *                   [batch][t_max][H*P] with FLAG_MAMBA1
  *   B               [batch][t_max][G_B][N] act dtype
  *   C               [batch][t_max][G_C][N] act dtype
  *   A               [H] float32, negative reals          D  [H] float32
+ *                   ([H*P][N] and [H*P] with FLAG_MAMBA1)
  *   n_prev_accepted [batch] int32, or null to use what the last mamba_spec_commit recorded
  *                   (zeros before any commit).  Values outside [0, min(k_max, t_max-k_draft)]
  *                   are clamped on the device and flagged in the status word.
@@ -141,7 +159,9 @@ int mamba_spec_verify(mamba_spec_ctx *ctx, void *state, void *conv_state, const 
 
 /* Algorithm 2's "j <- k'": records accept_len[b] (device, [batch], each in
  * [0, k_draft of the last verify]) as the next call's n_prev_accepted.  Moves no
- * state: the cache advances lazily, as the replay prefix of the next verify. */
+ * state: the cache advances lazily, as the replay prefix of the next verify.
+ * With FLAG_COMMIT_SELECTS a fully accepted sequence switches to the buffer that
+ * holds h_k instead and has nothing pending (see the flag). */
 int mamba_spec_commit(mamba_spec_ctx *ctx, const int32_t *accept_len, int32_t batch, void *stream);
 
 /* Same computation with the per-step tensors in HOST memory (pinned memory
@@ -191,6 +211,11 @@ int mamba_spec_status(mamba_spec_ctx *ctx, int32_t *device_flags_out);
  * would use) to HOST memory; with state and conv_state this is a complete
  * checkpoint of a layer stack.  Synchronises. */
 int mamba_spec_get_n_prev(mamba_spec_ctx *ctx, int32_t *n_prev_host, int32_t batch);
+
+/* FLAG_COMMIT_SELECTS: copies to HOST memory, for each of the first `batch` sequences, 0 if its cache is in
+ * (state, conv_state) and 1 if it is in (io->state_k, io->conv_state_k).  The same for every layer that
+ * shares the context, since all layers see the same commits.  Synchronises. */
+int mamba_spec_get_selection(mamba_spec_ctx *ctx, int32_t *sel_host, int32_t batch);
 
 /* Number of kernels this context has launched so far (HOST counter). */
 int64_t mamba_spec_launch_count(const mamba_spec_ctx *ctx);

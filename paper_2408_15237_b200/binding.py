@@ -24,6 +24,7 @@ lib = ctypes.CDLL(str(_LIB_PATH))
 OK = 0
 DTYPE_F32, DTYPE_BF16 = 0, 1
 FLAG_GATE, FLAG_CONV_SILU, FLAG_Y_F32, FLAG_STATE_K = 1, 2, 4, 8
+FLAG_MAMBA1, FLAG_DT_SOFTPLUS, FLAG_COMMIT_SELECTS = 16, 32, 64
 STATUS_NPREV_CLAMPED, STATUS_ACCEPT_CLAMPED, STATUS_COPY_TIMEOUT = 1, 2, 4
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_STREAM = 0, 1, 2
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_MISALIGNED, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOT_INIT = -1, -2, -3, -4, -5, -6
@@ -39,7 +40,7 @@ class IO(ctypes.Structure):
     _fields_ = [("conv_w", ctypes.c_void_p), ("conv_b", ctypes.c_void_p), ("z", ctypes.c_void_p),
                 ("y", ctypes.c_void_p), ("batch", ctypes.c_int32), ("layer", ctypes.c_int32),
                 ("t_max", ctypes.c_int32), ("stream", ctypes.c_void_p), ("state_k", ctypes.c_void_p),
-                ("conv_state_k", ctypes.c_void_p)]
+                ("conv_state_k", ctypes.c_void_p), ("dt_bias", ctypes.c_void_p)]
 
 
 _vp, _i32 = ctypes.c_void_p, ctypes.c_int32
@@ -57,6 +58,8 @@ lib.mamba_spec_status.restype = ctypes.c_int
 lib.mamba_spec_status.argtypes = [_vp, ctypes.POINTER(_i32)]
 lib.mamba_spec_get_n_prev.restype = ctypes.c_int
 lib.mamba_spec_get_n_prev.argtypes = [_vp, ctypes.POINTER(_i32), _i32]
+lib.mamba_spec_get_selection.restype = ctypes.c_int
+lib.mamba_spec_get_selection.argtypes = [_vp, ctypes.POINTER(_i32), _i32]
 lib.mamba_spec_launch_count.restype = ctypes.c_int64
 lib.mamba_spec_launch_count.argtypes = [_vp]
 lib.mamba_spec_last_kernel.restype = ctypes.c_char_p
@@ -132,6 +135,12 @@ def mamba_spec_get_n_prev(ctx, batch):
     return list(buf)
 
 
+def mamba_spec_get_selection(ctx, batch):
+    buf = (_i32 * batch)()
+    _check(ctx, lib.mamba_spec_get_selection(ctx, buf, batch))
+    return list(buf)
+
+
 def mamba_spec_launch_count(ctx) -> int:
     return lib.mamba_spec_launch_count(ctx)
 
@@ -169,24 +178,27 @@ class Verifier:
         except Exception:
             pass
 
-    def _io(self, conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k=None, conv_state_k=None):
+    def _io(self, conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k=None, conv_state_k=None, dt_bias=None):
         if stream is None:
             stream = torch.cuda.current_stream().cuda_stream
         return IO(_ptr(conv_w), _ptr(conv_b), _ptr(z), _ptr(y), batch, layer, t_max, stream, _ptr(state_k),
-                  _ptr(conv_state_k))
+                  _ptr(conv_state_k), _ptr(dt_bias))
 
     def verify(self, state, conv_state, x, dt, B, C, A, D, conv_w, conv_b, z, y, n_prev, k, layer=0, stream=None,
-               state_k=None, conv_state_k=None):
+               state_k=None, conv_state_k=None, dt_bias=None):
         c = self.cfg
         batch, t_max = x.shape[0], x.shape[1]
+        m1 = bool(c.flags & FLAG_MAMBA1)
+        chan = c.n_heads * c.head_dim
         want = {
             "state": (state, torch.float32, (batch, c.n_heads, c.head_dim, c.d_state)),
             "conv_state": (conv_state, self.act_dtype, (batch, c.conv_width - 1, c.n_heads * c.head_dim)),
             "x": (x, self.act_dtype, (batch, t_max, c.n_heads, c.head_dim)),
-            "dt": (dt, self.act_dtype, (batch, t_max, c.n_heads)),
+            "dt": (dt, self.act_dtype, (batch, t_max, chan if m1 else c.n_heads)),
             "B": (B, self.act_dtype, (batch, t_max, c.n_groups_b, c.d_state)),
             "C": (C, self.act_dtype, (batch, t_max, c.n_groups_c, c.d_state)),
-            "A": (A, torch.float32, (c.n_heads,)), "D": (D, torch.float32, (c.n_heads,)),
+            "A": (A, torch.float32, (chan, c.d_state) if m1 else (c.n_heads,)),
+            "D": (D, torch.float32, (chan,) if m1 else (c.n_heads,)),
             "conv_w": (conv_w, torch.float32, (c.n_heads * c.head_dim, c.conv_width)),
             "conv_b": (conv_b, torch.float32, (c.n_heads * c.head_dim,)),
             "y": (y, torch.float32 if c.flags & FLAG_Y_F32 else self.act_dtype, (batch, t_max, c.n_heads, c.head_dim)),
@@ -202,7 +214,14 @@ class Verifier:
             if not t.is_cuda or t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
                 raise ValueError(f"{name}: want contiguous CUDA {dtype} {shape}, got {t.dtype} {tuple(t.shape)} "
                                  f"cuda={t.is_cuda} contiguous={t.is_contiguous()}")
-        io = self._io(conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k, conv_state_k)
+        if dt_bias is not None:
+            want["dt_bias"] = (dt_bias, torch.float32, (chan,) if m1 else (c.n_heads,))
+        for name in ("dt_bias",):
+            if name in want:
+                t, dtype, shape = want[name]
+                if not t.is_cuda or t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
+                    raise ValueError(f"{name}: want contiguous CUDA {dtype} {shape}")
+        io = self._io(conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k, conv_state_k, dt_bias)
         mamba_spec_verify(self.ctx, state, conv_state, x, dt, B, C, A, D, n_prev, k, io)
 
     def commit(self, accept_len, stream=None):
@@ -212,6 +231,9 @@ class Verifier:
 
     def status(self) -> int:
         return mamba_spec_status(self.ctx)
+
+    def selection(self, batch):
+        return mamba_spec_get_selection(self.ctx, batch)
 
     @property
     def last_kernel(self) -> str:

@@ -15,15 +15,17 @@ struct VerifyParams {
     float *state;            // [batch][H][P][N]
     void *conv_state;        // [batch][W-1][H*P] act dtype
     const void *x;           // [batch][t_max][H][P]
-    const void *dt;          // [batch][t_max][H]
+    const void *dt;          // [batch][t_max][H]; Mamba-1 form: [batch][t_max][H*P]
     const void *B;           // [batch][t_max][GB][N]
     const void *C;           // [batch][t_max][GC][N]
     const void *z;           // [batch][t_max][H][P] or null
     void *y;                 // [batch][t_max][H][P]
     float *state_k;          // [batch][H][P][N], second snapshot (after all tokens), or null
     void *conv_state_k;      // [batch][W-1][H*P] act dtype, second snapshot, or null
-    const float *A;          // [H]
-    const float *D;          // [H]
+    const float *A;          // [H]; Mamba-1 form: [H*P][N]
+    const float *D;          // [H]; Mamba-1 form: [H*P]
+    const float *dt_bias;    // [H] ([H*P] in the Mamba-1 form) or null: added to the raw interval before its softplus
+    const int32_t *sel;      // [batch] or null: which of (state, state_k) holds each sequence's cache (commit-selects mode)
     const float *conv_w;     // [H*P][W]
     const float *conv_b;     // [H*P]
     const int32_t *n_prev;   // [batch]
@@ -38,11 +40,17 @@ constexpr int kFlagGate = 1;
 constexpr int kFlagConvSilu = 2;
 constexpr int kFlagYF32 = 4;
 constexpr int kFlagStateK = 8;
+constexpr int kFlagMamba1 = 16;        // interval per channel, A per (channel, state column), D per channel
+constexpr int kFlagDtSoftplus = 32;    // dt arrives raw: softplus(dt + dt_bias) is taken in the kernel
+constexpr int kFlagCommitSelects = 64; // the cache of sequence b is state or state_k as sel[b] says
+constexpr int kFlagYNewOnly = 1 << 16; // internal: y holds only the k new rows of each sequence, [batch][k]
 constexpr int kStatusNprevClamped = 1;
 constexpr int kStatusAcceptClamped = 2;
 constexpr int kStatusCopyTimeout = 4;
 
 __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + expf(-v)); }
+// softplus, the identity where exp would overflow into it anyway
+__device__ __forceinline__ float softplus_f(float v) { return v > 20.f ? v : log1pf(expf(v)); }
 
 __device__ __forceinline__ float ld_act(const float *p, size_t i) { return p[i]; }
 __device__ __forceinline__ float ld_act(const __nv_bfloat16 *p, size_t i) { return __bfloat162float(p[i]); }
@@ -89,6 +97,7 @@ struct alignas(64) InputMaps {
     TensorMapBytes x, z, B, C, dt, cst;
     TensorMapBytes state;    // [32 columns][rows][N/32 quarters], 128-byte swizzle
     TensorMapBytes state_k;  // the same over the second snapshot's buffer (FLAG_STATE_K only)
+    TensorMapBytes cst_k;    // the conv window of the second pair of buffers (commit-selects mode)
 };
 StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, size_t smem_per_block_optin);
 // Encodes the tensor maps of a launch (host work: eight driver calls); false if the driver refuses.

@@ -18,7 +18,7 @@ using namespace mspec;
 // buffers round after round, and encoding eight maps costs more host time than the launch itself.
 // A map depends only on addresses and shapes, so an entry stays valid for as long as its key matches.
 struct MapKey {
-    const void *state, *conv_state, *x, *dt, *B, *C, *z, *state_k;
+    const void *state, *conv_state, *x, *dt, *B, *C, *z, *state_k, *conv_state_k;
     int32_t batch, t_max, tcap, variant;
     bool operator==(const MapKey &o) const { return memcmp(this, &o, sizeof(MapKey)) == 0; }
 };
@@ -35,6 +35,7 @@ struct mamba_spec_ctx {
     size_t smem_per_sm = 0, smem_optin = 0;
     int32_t *d_n_prev = nullptr;  // [batch_max] pending n_prev recorded by commit
     int32_t *d_status = nullptr;  // one word
+    int32_t *d_sel = nullptr;     // [batch_max] which buffer holds each sequence's cache (FLAG_COMMIT_SELECTS)
     // device staging for mamba_spec_verify_host, allocated on its first use
     void *st_x = nullptr, *st_dt = nullptr, *st_B = nullptr, *st_C = nullptr, *st_z = nullptr, *st_y = nullptr;
     int32_t *st_n_prev = nullptr;
@@ -46,6 +47,9 @@ struct mamba_spec_ctx {
     std::string err;
     char last_kernel[112] = "none";
 };
+
+constexpr int kAllFlags = MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K |
+                          MAMBA_SPEC_FLAG_MAMBA1 | MAMBA_SPEC_FLAG_DT_SOFTPLUS | MAMBA_SPEC_FLAG_COMMIT_SELECTS;
 
 static thread_local std::string g_init_error;
 
@@ -102,13 +106,19 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 size_t act_bytes(const mamba_spec_config &c) { return c.act_dtype == MAMBA_SPEC_DTYPE_BF16 ? 2 : 4; }
 
-__global__ void commit_kernel(int32_t *n_prev, const int32_t *accept_len, int batch, int k, int32_t *status) {
+// Algorithm 2's choice of the state to keep: with `sel` a fully accepted sequence takes the buffer that holds
+// the state after all tokens (h_k) and has nothing pending; every other sequence keeps h_j and replays.
+__global__ void commit_kernel(int32_t *n_prev, const int32_t *accept_len, int batch, int k, int32_t *status, int32_t *sel) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     int a = accept_len[b];
     if (a < 0 || a > k) {
         atomicOr(status, kStatusAcceptClamped);
         a = a < 0 ? 0 : k;
+    }
+    if (sel != nullptr && a == k) {
+        sel[b] ^= 1;
+        a = 0;
     }
     n_prev[b] = a;
 }
@@ -135,10 +145,12 @@ int mamba_spec_init(const mamba_spec_config *cfg, mamba_spec_ctx **out) {
     if (c.k_max < 0 || c.k_max > 32) return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: k_max %d outside 0..32", c.k_max);
     if (c.act_dtype != MAMBA_SPEC_DTYPE_F32 && c.act_dtype != MAMBA_SPEC_DTYPE_BF16)
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: unknown act_dtype %d", c.act_dtype);
-    if (c.flags & ~(MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K))
+    if (c.flags & ~(kAllFlags))
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: unknown flag bits 0x%x", c.flags);
     if (c.kernel_select < 0 || c.kernel_select > MAMBA_SPEC_KERNEL_STREAM)
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: unknown kernel_select %d", c.kernel_select);
+    if ((c.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS) && !(c.flags & MAMBA_SPEC_FLAG_STATE_K))
+        return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: FLAG_COMMIT_SELECTS needs FLAG_STATE_K");
     // conv_state rows and token rows must keep 16-byte alignment per (sequence, row)
     if ((size_t)c.n_heads * c.head_dim * act_bytes(c) % 16)
         return fail(nullptr, MAMBA_SPEC_ERR_BAD_SHAPE, "init: H*P*sizeof(act) must be a multiple of 16 bytes");
@@ -165,11 +177,14 @@ int mamba_spec_init(const mamba_spec_config *cfg, mamba_spec_ctx **out) {
         e = cudaMalloc(&ctx->d_n_prev, sizeof(int32_t) * (size_t)c.batch_max);
     }
     if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_sel, sizeof(int32_t) * (size_t)c.batch_max);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_sel, 0, sizeof(int32_t) * (size_t)c.batch_max);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_n_prev, 0, sizeof(int32_t) * (size_t)c.batch_max);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int32_t));
     if (e != cudaSuccess) {
         cudaFree(ctx->d_n_prev);
         cudaFree(ctx->d_status);
+        cudaFree(ctx->d_sel);
         delete ctx;
         return fail(nullptr, MAMBA_SPEC_ERR_CUDA, "init: %s", cudaGetErrorString(e));
     }
@@ -201,6 +216,7 @@ static int check_and_fill(mamba_spec_ctx *ctx, VerifyParams &p, void *state, voi
     if ((c.flags & MAMBA_SPEC_FLAG_STATE_K) && (io->state_k == state || io->conv_state_k == conv_state))
         return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "%s: the second snapshot must not alias the cache", who);
     const void *ptrs[] = {state, conv_state, x, dt, B, C, A, D, io->conv_w, io->conv_b, io->z, io->y,
+                          (c.flags & MAMBA_SPEC_FLAG_DT_SOFTPLUS) ? (const void *)io->dt_bias : nullptr,
                           (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? io->state_k : nullptr,
                           (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? io->conv_state_k : nullptr};
     for (const void *q : ptrs)
@@ -209,6 +225,8 @@ static int check_and_fill(mamba_spec_ctx *ctx, VerifyParams &p, void *state, voi
     p.conv_state = conv_state;
     p.x = x; p.dt = dt; p.B = B; p.C = C; p.z = (c.flags & MAMBA_SPEC_FLAG_GATE) ? io->z : nullptr; p.y = io->y;
     p.A = A; p.D = D; p.conv_w = io->conv_w; p.conv_b = io->conv_b;
+    p.dt_bias = (c.flags & MAMBA_SPEC_FLAG_DT_SOFTPLUS) ? io->dt_bias : nullptr;
+    p.sel = (c.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS) ? ctx->d_sel : nullptr;
     p.state_k = (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? (float *)io->state_k : nullptr;
     p.conv_state_k = (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? io->conv_state_k : nullptr;
     p.n_prev = n_prev ? n_prev : ctx->d_n_prev;
@@ -232,7 +250,7 @@ static int launch(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t strea
             MapKey key;
             memset(&key, 0, sizeof key);
             key.state = p.state; key.conv_state = p.conv_state; key.x = p.x; key.dt = p.dt; key.B = p.B; key.C = p.C;
-            key.z = p.z; key.state_k = p.state_k; key.batch = p.batch; key.t_max = p.t_max; key.tcap = plan.layout.TCAP;
+            key.z = p.z; key.state_k = p.state_k; key.conv_state_k = p.conv_state_k; key.batch = p.batch; key.t_max = p.t_max; key.tcap = plan.layout.TCAP;
             key.variant = plan.variant;
             MapEntry *slot = nullptr;
             if (!ctx->map_cache.empty()) {
@@ -292,7 +310,8 @@ int mamba_spec_commit(mamba_spec_ctx *ctx, const int32_t *accept_len, int32_t ba
     if (!guard.ok) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "commit: cannot select device %d", ctx->cfg.device);
     const int k = ctx->last_k >= 0 ? ctx->last_k : ctx->cfg.k_max;
     cudaStream_t s = (cudaStream_t)stream;
-    commit_kernel<<<(batch + 127) / 128, 128, 0, s>>>(ctx->d_n_prev, accept_len, batch, k, ctx->d_status);
+    commit_kernel<<<(batch + 127) / 128, 128, 0, s>>>(ctx->d_n_prev, accept_len, batch, k, ctx->d_status,
+                                                      (ctx->cfg.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS) ? ctx->d_sel : nullptr);
     CUDA_TRY(ctx, cudaGetLastError());
     ctx->launches++;
     ctx->last_stream = s;
@@ -314,7 +333,7 @@ int mamba_spec_verify_host(mamba_spec_ctx *ctx, void *state, void *conv_state, c
     DeviceGuard guard(c.device);
     if (!guard.ok) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "verify_host: cannot select device %d", c.device);
     const size_t ab = act_bytes(c), rows = (size_t)c.batch_max * t_cap;
-    const size_t n_x = rows * c.n_heads * c.head_dim * ab, n_dt = rows * c.n_heads * ab;
+    const size_t n_x = rows * c.n_heads * c.head_dim * ab, n_dt = (c.flags & MAMBA_SPEC_FLAG_MAMBA1) ? n_x : rows * c.n_heads * ab;
     const size_t n_B = rows * c.n_groups_b * c.d_state * ab, n_C = rows * c.n_groups_c * c.d_state * ab;
     if (!ctx->staging_ready) {   // all or nothing: a failed allocation leaves no half-built staging behind
         void **slots[] = {&ctx->st_x, &ctx->st_z, &ctx->st_y, &ctx->st_dt, &ctx->st_B, &ctx->st_C, (void **)&ctx->st_n_prev};
@@ -341,7 +360,7 @@ int mamba_spec_verify_host(mamba_spec_ctx *ctx, void *state, void *conv_state, c
     const size_t used = (size_t)io->batch * io->t_max;
     const size_t b_x = used * c.n_heads * c.head_dim * ab;
     CUDA_TRY(ctx, cudaMemcpyAsync(ctx->st_x, x_host, b_x, cudaMemcpyHostToDevice, s));
-    CUDA_TRY(ctx, cudaMemcpyAsync(ctx->st_dt, dt_host, used * c.n_heads * ab, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(ctx, cudaMemcpyAsync(ctx->st_dt, dt_host, (c.flags & MAMBA_SPEC_FLAG_MAMBA1) ? b_x : used * c.n_heads * ab, cudaMemcpyHostToDevice, s));
     CUDA_TRY(ctx, cudaMemcpyAsync(ctx->st_B, B_host, used * c.n_groups_b * c.d_state * ab, cudaMemcpyHostToDevice, s));
     CUDA_TRY(ctx, cudaMemcpyAsync(ctx->st_C, C_host, used * c.n_groups_c * c.d_state * ab, cudaMemcpyHostToDevice, s));
     if (c.flags & MAMBA_SPEC_FLAG_GATE) CUDA_TRY(ctx, cudaMemcpyAsync(ctx->st_z, io->z, b_x, cudaMemcpyHostToDevice, s));
@@ -366,9 +385,11 @@ static int verify_host_static_impl(mamba_spec_ctx *tmp, void *state, void *conv_
         c.conv_width < 1 || c.conv_width > kMaxConvWidth || c.n_groups_b < 1 || c.n_groups_c < 1 ||
         c.n_heads % c.n_groups_b || c.n_heads % c.n_groups_c || c.k_max < 0 || c.k_max > 32 ||
         (c.act_dtype != MAMBA_SPEC_DTYPE_F32 && c.act_dtype != MAMBA_SPEC_DTYPE_BF16) ||
-        (c.flags & ~(MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K)) || c.kernel_select < 0 ||
+        (c.flags & ~(kAllFlags)) || c.kernel_select < 0 ||
         c.kernel_select > MAMBA_SPEC_KERNEL_STREAM || ((size_t)c.n_heads * c.head_dim * act_bytes(c)) % 16)
         return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: configuration rejected (same rules as mamba_spec_init)");
+    if (c.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS)
+        return fail(tmp, MAMBA_SPEC_ERR_UNSUPPORTED, "verify_host_static: FLAG_COMMIT_SELECTS needs a context");
     if (!io) return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: io is null");
     if (!x_host || !dt_host || !B_host || !C_host || !n_prev_host || !io->y)
         return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: a required host pointer is null");
@@ -393,7 +414,7 @@ static int verify_host_static_impl(mamba_spec_ctx *tmp, void *state, void *conv_
     }
     // carve the staging array: pending lengths, status word, then the token slabs
     const size_t ab = act_bytes(c), used = (size_t)io->batch * io->t_max;
-    const size_t b_x = used * c.n_heads * c.head_dim * ab, b_dt = used * c.n_heads * ab;
+    const size_t b_x = used * c.n_heads * c.head_dim * ab, b_dt = (c.flags & MAMBA_SPEC_FLAG_MAMBA1) ? b_x : used * c.n_heads * ab;
     const size_t b_B = used * c.n_groups_b * c.d_state * ab, b_C = used * c.n_groups_c * c.d_state * ab;
     const size_t b_y = (c.flags & MAMBA_SPEC_FLAG_Y_F32) ? b_x / ab * 4 : b_x;
     // every factor is a positive int32, so no single product above can wrap a 64-bit size_t unless it is far
@@ -477,6 +498,18 @@ int mamba_spec_get_n_prev(mamba_spec_ctx *ctx, int32_t *n_prev_host, int32_t bat
     return MAMBA_SPEC_OK;
 }
 
+int mamba_spec_get_selection(mamba_spec_ctx *ctx, int32_t *sel_host, int32_t batch) {
+    if (!ctx) return fail(nullptr, MAMBA_SPEC_ERR_NOT_INIT, "get_selection: ctx is null");
+    if (!sel_host) return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "get_selection: output pointer is null");
+    if (batch < 1 || batch > ctx->cfg.batch_max)
+        return fail(ctx, MAMBA_SPEC_ERR_BAD_SHAPE, "get_selection: batch %d outside 1..%d", batch, ctx->cfg.batch_max);
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "get_selection: cannot select device %d", ctx->cfg.device);
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->last_stream));
+    CUDA_TRY(ctx, cudaMemcpy(sel_host, ctx->d_sel, sizeof(int32_t) * (size_t)batch, cudaMemcpyDeviceToHost));
+    return MAMBA_SPEC_OK;
+}
+
 int64_t mamba_spec_launch_count(const mamba_spec_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 const char *mamba_spec_last_kernel(const mamba_spec_ctx *ctx) { return ctx ? ctx->last_kernel : "none"; }
@@ -489,7 +522,7 @@ void mamba_spec_destroy(mamba_spec_ctx *ctx) {
         DeviceGuard guard(ctx->cfg.device);
         if (guard.ok) {
             cudaDeviceSynchronize();
-            void *bufs[] = {ctx->d_n_prev, ctx->d_status, ctx->st_x, ctx->st_dt, ctx->st_B, ctx->st_C,
+            void *bufs[] = {ctx->d_n_prev, ctx->d_status, ctx->d_sel, ctx->st_x, ctx->st_dt, ctx->st_B, ctx->st_C,
                             ctx->st_z, ctx->st_y, ctx->st_n_prev};
             for (void *b : bufs)
                 if (b) cudaFree(b);

@@ -11,11 +11,17 @@
 // store y.  After token j_b-1 the row and the conv window are written back;
 // the k draft tokens that follow only ever touch registers (Sec. 4.2: the
 // snapshot h_j is saved before the drafts are evaluated; Sec. 4.3 i)-iii)).
+//
+// The same kernel covers the variants of the parameterisation: the Mamba-1 form
+// (Algorithm 1: interval per channel, A per channel and state column, where the
+// decay is an exp per state element), the softplus of a raw interval taken in the
+// kernel, the mode in which each sequence's cache is one of two buffers
+// (Algorithm 2 keeps h_j or h_k), and outputs for the new rows only.
 #include "common.cuh"
 
 namespace mspec {
 
-template <typename act_t>
+template <typename act_t, bool M1>
 __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams p) {
     const int lane = threadIdx.x & 31;
     const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -32,7 +38,12 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
     const int Cch = H * P, c = h * P + pr;
     const act_t *x = (const act_t *)p.x, *dt = (const act_t *)p.dt, *Bm = (const act_t *)p.B,
                 *Cm = (const act_t *)p.C, *z = (const act_t *)p.z;
-    act_t *y = (act_t *)p.y, *cst = (act_t *)p.conv_state;
+    act_t *y = (act_t *)p.y;
+    // commit-selects mode: this sequence's cache is the second pair of buffers when sel says so; the state
+    // at the verified position goes back to where the cache is, the state after all tokens to the other pair
+    const bool swapped = p.sel != nullptr && p.sel[b] != 0;
+    act_t *cst = (act_t *)(swapped ? p.conv_state_k : p.conv_state), *cst_other = (act_t *)(swapped ? p.conv_state : p.conv_state_k);
+    float *st_cur = swapped ? p.state_k : p.state, *st_other = swapped ? p.state : p.state_k;
     const int gB = h / (H / p.GB), gC = h / (H / p.GC);
 
     float win[kMaxConvWidth - 1], tap[kMaxConvWidth];
@@ -41,11 +52,18 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
         win[w] = (w < W - 1) ? ld_act(cst, ((size_t)b * (W - 1) + w) * Cch + c) : 0.f;
 #pragma unroll
     for (int w = 0; w < kMaxConvWidth; ++w) tap[w] = (w < W) ? p.conv_w[(size_t)c * W + w] : 0.f;
-    const float bias = p.conv_b[c], A_h = p.A[h], D_h = p.D[h];
+    const float bias = p.conv_b[c], A_h = M1 ? 0.f : p.A[h], D_h = p.D[M1 ? c : h];
+    const bool sp = (p.flags & kFlagDtSoftplus) != 0, y_new = (p.flags & kFlagYNewOnly) != 0;
+    const float dtb = (sp && p.dt_bias) ? p.dt_bias[M1 ? c : h] : 0.f;
 
     constexpr int kRegs = kMaxStateDim / 32;
     float hreg[kRegs];
-    float *srow = p.state + (size_t)row * N;
+    float *srow = st_cur + (size_t)row * N;
+    float Areg[M1 ? kRegs : 1];   // Mamba-1 form: this channel's row of A
+    if (M1) {
+#pragma unroll
+        for (int i = 0; i < kRegs; ++i) Areg[M1 ? i : 0] = (lane + 32 * i < N) ? p.A[(size_t)c * N + lane + 32 * i] : 0.f;
+    }
 #pragma unroll
     for (int i = 0; i < kRegs; ++i) hreg[i] = (lane + 32 * i < N) ? srow[lane + 32 * i] : 0.f;
 
@@ -67,15 +85,16 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
         for (int w = 0; w < kMaxConvWidth - 1; ++w)
             if (w == W - 2) win[w] = xin;
 
-        const float dtv = ld_act(dt, bt * H + h);
-        const float a = expf(dtv * A_h), u = dtv * xc;
+        float dtv = ld_act(dt, M1 ? bt * Cch + c : bt * H + h);
+        if (sp) dtv = softplus_f(dtv + dtb);
+        const float a = M1 ? 0.f : expf(dtv * A_h), u = dtv * xc;
         const act_t *Bv = Bm + (bt * p.GB + gB) * N, *Cv = Cm + (bt * p.GC + gC) * N;
         float part = 0.f;
 #pragma unroll
         for (int i = 0; i < kRegs; ++i) {
             const int n = lane + 32 * i;
             if (n < N) {
-                hreg[i] = fmaf(a, hreg[i], u * ld_act(Bv, n));
+                hreg[i] = fmaf(M1 ? expf(dtv * Areg[M1 ? i : 0]) : a, hreg[i], u * ld_act(Bv, n));
                 part = fmaf(ld_act(Cv, n), hreg[i], part);
             }
         }
@@ -84,8 +103,12 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
         if (lane == 0) {
             float v = fmaf(D_h, xc, part);
             if ((p.flags & kFlagGate) && z) v *= silu_f(ld_act(z, (bt * H + h) * P + pr));
-            if (p.flags & kFlagYF32) reinterpret_cast<float *>(p.y)[(bt * H + h) * P + pr] = v;
-            else st_act(y, (bt * H + h) * P + pr, v);
+            // (with new rows only: y is [batch][k], the replayed rows' outputs are dropped)
+            const size_t yi = y_new ? (((size_t)b * p.k + (t - j)) * H + h) * P + pr : (bt * H + h) * P + pr;
+            if (!y_new || t >= j) {
+                if (p.flags & kFlagYF32) reinterpret_cast<float *>(p.y)[yi] = v;
+                else st_act(y, yi, v);
+            }
         }
         if (t == j - 1) {  // the newly verified position: cache the state and the conv window here
 #pragma unroll
@@ -99,12 +122,12 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
         }
     }
     if (p.state_k) {  // second snapshot: the cache after all T tokens (Algorithm 2: h_k)
-        float *krow = p.state_k + (size_t)row * N;
+        float *krow = st_other + (size_t)row * N;
 #pragma unroll
         for (int i = 0; i < kRegs; ++i)
             if (lane + 32 * i < N) krow[lane + 32 * i] = hreg[i];
         if (lane == 0) {
-            act_t *cstk = (act_t *)p.conv_state_k;
+            act_t *cstk = cst_other;
 #pragma unroll
             for (int w = 0; w < kMaxConvWidth - 1; ++w)
                 if (w < W - 1) st_act(cstk, ((size_t)b * (W - 1) + w) * Cch + c, win[w]);
@@ -117,10 +140,11 @@ cudaError_t launch_verify_generic(const VerifyParams &p, bool bf16, cudaStream_t
     const int warps_per_block = 4;
     const long long blocks = (rows + warps_per_block - 1) / warps_per_block;
     if (blocks <= 0 || blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    if (bf16)
-        verify_generic_kernel<__nv_bfloat16><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
-    else
-        verify_generic_kernel<float><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
+    const bool m1 = (p.flags & kFlagMamba1) != 0;
+    if (bf16 && m1) verify_generic_kernel<__nv_bfloat16, true><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
+    else if (bf16) verify_generic_kernel<__nv_bfloat16, false><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
+    else if (m1) verify_generic_kernel<float, true><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
+    else verify_generic_kernel<float, false><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

@@ -262,7 +262,9 @@ __device__ __forceinline__ bool issue_raw(const VerifyParams &p, const StreamLay
         const int cy = lane == 5 ? b * (kW - 1) : row0;
         const uint32_t dst = raw + (lane == 0 ? L.r_x : lane == 1 ? L.r_z : lane == 2 ? L.r_B : lane == 3 ? L.r_C
                                                                    : lane == 4 ? L.r_dt : L.r_cst);
-        if (lane != 1 || p.z != nullptr) tma_load_2d(dst, as_map(&tm.x + lane), cx, cy, bar);
+        // (commit-selects mode: the conv window comes from whichever buffer holds this sequence's cache)
+        const TensorMapBytes *map = (lane == 5 && p.sel != nullptr && p.sel[b] != 0) ? &tm.cst_k : &tm.x + lane;
+        if (lane != 1 || p.z != nullptr) tma_load_2d(dst, as_map(map), cx, cy, bar);
     } else if (lane < 8) {
         const bool taps = lane == 6;
         bulk_g2s(raw + (taps ? L.r_cw : L.r_cb), taps ? (const void *)(p.conv_w + (size_t)c0 * kW) : (const void *)(p.conv_b + c0),
@@ -303,7 +305,8 @@ __device__ __forceinline__ void producer_role(const VerifyParams &p, const Strea
                 const uint32_t sbar = smem_u32(&ctl.state_full[ss]);
                 ctl.state_par[ss] = sp;
                 mbar_arrive_expect_tx(sbar, kStateBytes);
-                tma_load_3d(smem_base + L.state_off + ss * L.state_stride, as_map(&tm.state), 0, ps.q * CR, 0, sbar);
+                const bool swapped = p.sel != nullptr && p.sel[ps.b] != 0;   // commit-selects mode: where this sequence's cache is
+                tma_load_3d(smem_base + L.state_off + ss * L.state_stride, as_map(swapped ? &tm.state_k : &tm.state), 0, ps.q * CR, 0, sbar);
             }
         }
         advance(ps, wi.one, H, cph);
@@ -327,7 +330,7 @@ __device__ __forceinline__ void producer_role(const VerifyParams &p, const Strea
 template <int N, int CR, bool SNAP>
 __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const StreamLayout &L, const unsigned char *raw,
                                                unsigned char *gb, int b, int h, int rc, int j, int T,
-                                               float A_of_head, float D_of_head, int gtid) {
+                                               float A_of_head, float D_of_head, int gtid, bool swapped) {
     constexpr int HR = CR / 2;      // row pairs
     constexpr int CPR = N / 8;      // 16-byte pieces (8 bf16) per B or C row
     const int H = p.H, P = p.P;
@@ -337,6 +340,13 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
     float *Gm = reinterpret_cast<float *>(gb + L.c_G);    // [kMaxT][kMaxT], entries s <= t < T
     float *xcs = reinterpret_cast<float *>(gb + L.c_xc);  // [t][CR]
     const unsigned short *dtr = reinterpret_cast<const unsigned short *>(raw + L.r_dt) + (h & 7);   // dt_t at [t * 8]
+    // the sampling interval of token r: as it arrives, or softplus(raw + bias) when it arrives raw (Sec. 2.2)
+    const bool dt_raw = (p.flags & kFlagDtSoftplus) != 0;
+    const float dt_b = (dt_raw && p.dt_bias != nullptr) ? p.dt_bias[h] : 0.f;
+    auto dt_at = [&](int r) {
+        const float v = bf16_bits_to_f32(dtr[r * 8]);
+        return dt_raw ? softplus_f(v + dt_b) : v;
+    };
     const uint32_t *cs32 = reinterpret_cast<const uint32_t *>(raw + L.r_cst), *xs32 = reinterpret_cast<const uint32_t *>(raw + L.r_x);
 
     // ---- pairs, by the last warp: the T x T products C_t . B_s are a small bf16 matrix product, exact in
@@ -369,7 +379,7 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
             }
         }
         // lane r holds dt_r and E_r = sum_{r' <= r} dt_r'
-        const float dtv = lane < T ? bf16_bits_to_f32(dtr[lane * 8]) : 0.f;
+        const float dtv = lane < T ? dt_at(lane) : 0.f;
         float E = dtv;
 #pragma unroll
         for (int m = 1; m < kMaxT; m <<= 1) {
@@ -425,13 +435,13 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
         if (pw == 0)   // zero rows up to the next multiple of four tokens (read, times zero, by the output loop)
             for (int t = T; t < ((T + 3) & ~3); ++t) reinterpret_cast<float2 *>(xcs)[t * HR + lane] = make_float2(0.f, 0.f);
         if (j > 0 && pw < kW - 1) {  // the last W-1 inputs up to token j-1 become the cached window: warp i writes slot i
-            uint32_t *out = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned short *>(p.conv_state) +
+            uint32_t *out = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned short *>(swapped ? p.conv_state_k : p.conv_state) +
                                                          (size_t)b * (kW - 1) * (H * P) + h * P + rc * CR) + lane;
             const int tau = j - (kW - 1) + pw;
             out[(size_t)pw * (H * P / 2)] = tau < 0 ? cs32[(kW - 1 + tau) * HR + lane] : xs32[tau * HR + lane];
         }
         if (SNAP && pw < kW - 1) {  // second snapshot: the window after all T tokens
-            uint32_t *out = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned short *>(p.conv_state_k) +
+            uint32_t *out = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned short *>(swapped ? p.conv_state : p.conv_state_k) +
                                                          (size_t)b * (kW - 1) * (H * P) + h * P + rc * CR) + lane;
             const int tau = T - (kW - 1) + pw;
             out[(size_t)pw * (H * P / 2)] = tau < 0 ? cs32[(kW - 1 + tau) * HR + lane] : xs32[tau * HR + lane];
@@ -467,12 +477,12 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
         float sum = 0.f;   // every lane walks all T tokens (uniform broadcast loads, nothing to wait for in turn)
 #pragma unroll 4
         for (int r = 0; r < T; ++r) {
-            const float v = bf16_bits_to_f32(dtr[r * 8]);
+            const float v = dt_at(r);
             sum += (r >= lo && r < hi) ? v : 0.f;
         }
         const float ex = expf(A_of_head * sum);
         if (lane < T && lane < 16) hc->alpha[lane] = ex;
-        if (is_wsp) hc->wsp[lane - 16] = bf16_bits_to_f32(dtr[(lane - 16) * 8]) * ex;
+        if (is_wsp) hc->wsp[lane - 16] = dt_at(lane - 16) * ex;
         if (lane == 31) {
             hc->alpha_j = ex;
             hc->D = D_of_head;
@@ -482,11 +492,11 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
             float sum2 = 0.f;
 #pragma unroll 4
             for (int r = 0; r < T; ++r) {
-                const float v = bf16_bits_to_f32(dtr[r * 8]);
+                const float v = dt_at(r);
                 sum2 += (r >= lo2 && r < hi2) ? v : 0.f;
             }
             const float ex2 = expf(A_of_head * sum2);
-            if (lane < 16 && lane >= j && lane < T) hc->wspT[lane] = bf16_bits_to_f32(dtr[lane * 8]) * ex2;
+            if (lane < 16 && lane >= j && lane < T) hc->wspT[lane] = dt_at(lane) * ex2;
             if (lane == 31) hc->alpha_jT = ex2;
         }
     }
@@ -504,7 +514,7 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
 template <int N, int CR, bool SNAP>
 __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const StreamLayout &L, const InputMaps &tm,
                                              unsigned char *st, unsigned char *gb, uint32_t empty_bar, int bar_id, int q,
-                                             int b, int h, int rc, int j, int T, int gtid) {
+                                             int b, int h, int rc, int j, int T, int gtid, bool swapped) {
     constexpr int NQ = N / 32;                                  // column quarters of a row
     constexpr int RBK = kGroupWarps / NQ;                       // row blocks (warps per quarter)
     constexpr int RPT = (CR / (32 * RBK)) > 0 ? CR / (32 * RBK) : 1;  // rows per thread
@@ -593,7 +603,7 @@ __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const Stream
     }
     named_bar_sync(bar_id, kGroupThreads);   // partial sums and (if any) the new state are in shared memory
     if (j > 0 && gtid == 0) {
-        tma_store_3d(as_map(&tm.state), smem_u32(st), 0, q * CR, 0);
+        tma_store_3d(as_map(swapped ? &tm.state_k : &tm.state), smem_u32(st), 0, q * CR, 0);
         bulk_commit_group();
     }
     if (snap2) {
@@ -645,7 +655,7 @@ __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const Stream
         }
         named_bar_sync(bar_id, kGroupThreads);
         if (gtid == 0) {
-            tma_store_3d(as_map(&tm.state_k), smem_u32(st), 0, q * CR, 0);
+            tma_store_3d(as_map(swapped ? &tm.state : &tm.state_k), smem_u32(st), 0, q * CR, 0);
             bulk_commit_group();
         }
     }
@@ -727,20 +737,21 @@ __device__ __forceinline__ void compute_role(const VerifyParams &p, const Stream
     ring_advance(rs, rp, group, L.R);
     for (; it < nmine; it += L.ngroups) {
         const int j = pending_of(p, ctl, x.b), T = j + p.k;
+        const bool swapped = SNAP && p.sel != nullptr && p.sel[x.b] != 0;   // commit-selects mode: the cache is in the second buffers
         // the group's buffer is free once every warp has left the previous chunk; the inputs must be in
         bool ok = mbar_wait(smem_u32(&ctl.raw_full[rs]), (uint32_t)rp, &ctl.abort);
         ok = named_bar_and(bar_id, kGroupThreads, ok);
         if (!ok) break;
         if (store_pending) { release_stage(pending_bar); store_pending = false; }
         const unsigned char *raw = smem + L.raw_off + (size_t)rs * L.raw_stride;
-        prologue_phase<N, CR, SNAP>(p, L, raw, gb, x.b, x.h, x.rc, j, T, ctl.A[x.h], ctl.D[x.h], gtid);
+        prologue_phase<N, CR, SNAP>(p, L, raw, gb, x.b, x.h, x.rc, j, T, ctl.A[x.h], ctl.D[x.h], gtid, swapped);
         ok = mbar_wait(smem_u32(&ctl.state_full[ss]), (uint32_t)sp, &ctl.abort);
         ok = named_bar_and(bar_id, kGroupThreads, ok);   // also: the group's buffer is complete
         if (lane == 0) mbar_arrive(smem_u32(&ctl.raw_empty[rs]));
         if (!ok) break;
         unsigned char *st = smem + L.state_off + (size_t)ss * L.state_stride;
         pending_bar = smem_u32(&ctl.state_empty[ss]);
-        store_pending = stream_phase<N, CR, SNAP>(p, L, tm, st, gb, pending_bar, bar_id, x.q, x.b, x.h, x.rc, j, T, gtid);
+        store_pending = stream_phase<N, CR, SNAP>(p, L, tm, st, gb, pending_bar, bar_id, x.q, x.b, x.h, x.rc, j, T, gtid, swapped);
         advance(x, wi.grp, H, cph);
         ring_advance(ss, sp, L.ngroups, L.S);
         ring_advance(rs, rp, L.ngroups, L.R);
@@ -921,6 +932,8 @@ StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, si
         return plan;
     };
     if (!bf16) return reject("activations are not bf16");
+    if (p.flags & kFlagMamba1) return reject("the Mamba-1 parameterisation runs in the generic kernel");
+    if (p.flags & kFlagYNewOnly) return reject("variant not in the streaming kernel");
     if (p.W != kW) return reject("conv width is not 4");
     if (p.N != 64 && p.N != 128) return reject("state dim is not 64 or 128");
     if (p.P % 32) return reject("head dim is not a multiple of 32");
@@ -1022,8 +1035,12 @@ bool encode_stream_maps(const VerifyParams &p, const StreamPlan &plan, InputMaps
               encode_2d(fn, &tm->dt, p.dt, (size_t)p.H, rows, 8, L.TCAP) &&
               encode_2d(fn, &tm->cst, p.conv_state, hp, (size_t)p.batch * (kW - 1), CR, kW - 1) &&
               encode_state(fn, &tm->state, p.state, srows, p.N, CR);
-    if (p.state_k) ok = ok && encode_state(fn, &tm->state_k, p.state_k, srows, p.N, CR);
-    else memcpy(&tm->state_k, &tm->state, sizeof(TensorMapBytes));
+    if (p.state_k) ok = ok && encode_state(fn, &tm->state_k, p.state_k, srows, p.N, CR) &&
+                        encode_2d(fn, &tm->cst_k, p.conv_state_k, hp, (size_t)p.batch * (kW - 1), CR, kW - 1);
+    else {
+        memcpy(&tm->state_k, &tm->state, sizeof(TensorMapBytes));
+        memcpy(&tm->cst_k, &tm->cst, sizeof(TensorMapBytes));
+    }
     return ok;
 }
 

@@ -201,3 +201,28 @@ class Rounds:
 
 def with_batch(s: Shape, Bt: int) -> Shape:
     return replace(s, Bt=Bt, name=f"{s.name}_bt{Bt}")
+
+
+def m1_params(s: Shape, layer: int = 0):
+    """Mamba-1 form of the per-layer constants (Algorithm 1): A [H*P, N] negative, D [H*P]; fp32."""
+    g = rng(s.name, layer, "params_m1")
+    A = -np.exp(g.uniform(0.0, np.log(16.0), size=(s.H * s.P, s.N))).astype(np.float32)
+    D = g.standard_normal(s.H * s.P).astype(np.float32)
+    return A, D
+
+
+def m1_dt_stream(s: Shape, layer: int, length: int) -> np.ndarray:
+    """Mamba-1 form of the sampling intervals: one per (token, channel), [Bt, L, H*P], same distribution as dt."""
+    g = rng(s.name, layer, "stream_m1_dt", length)
+    pre = g.standard_normal((s.Bt, length, s.H * s.P), dtype=np.float32) - np.float32(2.0)
+    return to_act(np.log1p(np.exp(pre.astype(np.float64))).astype(np.float32), s.act)
+
+
+def raw_dt_stream(s: Shape, layer: int, length: int, per_channel: bool = False):
+    """Raw intervals (before the softplus) and their bias: dt_raw ~ N(0,1) in the activation precision, [Bt, L, H]
+    ([Bt, L, H*P] per channel), bias ~ N(-2, 0.25) fp32, so that softplus(dt_raw + bias) is distributed like dt."""
+    g = rng(s.name, layer, "stream_raw_dt", length, per_channel)
+    n = s.H * s.P if per_channel else s.H
+    raw = to_act(g.standard_normal((s.Bt, length, n), dtype=np.float32), s.act)
+    bias = (np.float32(-2.0) + np.float32(0.5) * g.standard_normal(n)).astype(np.float32)
+    return raw, bias

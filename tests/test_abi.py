@@ -59,7 +59,7 @@ def cfg(binding, **over):
 
 @pytest.mark.parametrize("over,code", [
     (dict(batch_max=0), -1), (dict(d_state=512), -4), (dict(conv_width=9), -4), (dict(n_groups_b=3), -2),
-    (dict(k_max=33), -1), (dict(act_dtype=7), -1), (dict(flags=16), -1), (dict(kernel_select=5), -1),
+    (dict(k_max=33), -1), (dict(act_dtype=7), -1), (dict(flags=1 << 12), -1), (dict(flags=64), -1), (dict(kernel_select=5), -1),
     (dict(n_heads=1, head_dim=4, n_groups_b=1, n_groups_c=1), -2),
 ])
 def test_init_rejects_bad_configurations_before_touching_a_device(binding, over, code):

@@ -1,0 +1,184 @@
+"""GPU parity of the parameterisation variants against the fp64 oracle, through the C ABI:
+the Mamba-1 form (Algorithm 1), the softplus of a raw interval taken in the kernel (Sec. 2.2), and
+Algorithm 2's choice between h_j and h_k made by commit (two buffers per sequence, no replay after a
+fully accepted round)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2408_15237_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+GENERIC, STREAM = 1, 2
+
+
+def H():
+    import harness
+    return harness
+
+
+M1_SMALL = synth.Shape("m1_small", Bt=3, H=4, P=16, N=32, GB=2, GC=4, W=4, k=3, act="fp32")
+M1_BF16 = synth.Shape("m1_bf16", Bt=2, H=8, P=64, N=128, GB=2, GC=8, W=4, k=4, act="bf16")
+
+
+@pytest.mark.parametrize("s,tol", [(M1_SMALL, 1e-5), (M1_BF16, 1e-5)])
+def test_mamba1_form_matches_the_oracle(s, tol):
+    """Interval per channel, A per (channel, state column), D per channel; y in float32 so that the only error
+    left is the kernel's fp32 arithmetic.  Three rounds with replay, then a flush."""
+    h = H()
+    from paper_2408_15237_b200 import binding
+    flags = s.flags | binding.FLAG_MAMBA1 | binding.FLAG_Y_F32
+    ver = binding.Verifier(s.Bt, s.H, s.P, s.N, s.GB, s.GC, s.W, s.k, act=s.act, flags=flags)
+    ad = h.act_dtype(s)
+    A, D = synth.m1_params(s)
+    _, _, cw, cb = synth.layer_params(s)
+    st, cv = synth.initial_cache(s)
+    L = 4 * s.k + 4
+    stream = synth.token_stream(s, 0, L)
+    stream["dt"] = synth.m1_dt_stream(s, 0, L)
+    r = synth.Rounds(s, stream, first_j=2)
+    o_state, o_conv = st.astype(np.float64), cv.astype(np.float64)
+    state, conv = h.dev(st, torch.float32), h.dev(cv, ad)
+    dA, dD, dcw, dcb = (h.dev(a, torch.float32) for a in (A, D, cw, cb))
+    for rd, k in enumerate([s.k, s.k, s.k, 0]):
+        b = r.batch(k=k)
+        t = {n: h.dev(b[n], ad) for n in ("x", "z", "dt", "B", "C")}
+        y = torch.full(t["x"].shape, float("nan"), device="cuda", dtype=torch.float32)
+        ver.verify(state, conv, t["x"], t["dt"], t["B"], t["C"], dA, dD, dcw, dcb, t["z"], y, h.dev(b["n_prev"], torch.int32), k)
+        torch.cuda.synchronize()
+        assert ver.last_kernel == "generic"
+        y_ref, o_state, o_conv = oracle.verify_m1(o_state, o_conv, b["x"], b["dt"], b["B"], b["C"], A, D, cw, cb, b["z"],
+                                                   b["n_prev"], k, s.flags, threads=oracle.host_threads())
+        yg = y.cpu().numpy().astype(np.float64)
+        valid = ~np.isnan(y_ref)
+        assert np.isnan(yg[~valid]).all() and not np.isnan(yg[valid]).any()
+        if valid.any():
+            assert h.rel_l2(yg[valid], y_ref[valid]) <= tol, f"round {rd}"
+        assert h.rel_l2(state.cpu().numpy(), o_state) <= tol, f"round {rd}"
+        assert np.abs(conv.float().cpu().numpy().astype(np.float64) - o_conv).max() == 0.0
+        if k:
+            r.accept(synth.acceptance(s, rd))
+    assert ver.status() == 0
+    ver.close()
+
+
+@pytest.mark.parametrize("s,kernel,m1", [(synth.CONFIGS[0], GENERIC, False), (M1_SMALL, GENERIC, True),
+                                         (synth.SWEEP[(4, 4)], STREAM, False), (synth.SWEEP[(4, 4)], GENERIC, False)])
+def test_softplus_of_the_raw_interval_in_the_kernel(s, kernel, m1):
+    """dt arrives raw with a bias; the kernel's softplus(dt + bias) against the oracle fed with the interval
+    computed on the host in fp64."""
+    h = H()
+    from paper_2408_15237_b200 import binding
+    flags = s.flags | binding.FLAG_DT_SOFTPLUS | binding.FLAG_Y_F32 | (binding.FLAG_MAMBA1 if m1 else 0)
+    ver = binding.Verifier(s.Bt, s.H, s.P, s.N, s.GB, s.GC, s.W, s.k, act=s.act, flags=flags, kernel=kernel)
+    ad = h.act_dtype(s)
+    A, D, cw, cb = synth.layer_params(s)
+    if m1:
+        A, D = synth.m1_params(s)
+    st, cv = synth.initial_cache(s)
+    L = 3 * s.k + 4
+    stream = synth.token_stream(s, 0, L)
+    raw, bias = synth.raw_dt_stream(s, 0, L, per_channel=m1)
+    stream["dt"] = raw
+    r = synth.Rounds(s, stream, first_j=min(2, s.k))
+    o_state, o_conv = st.astype(np.float64), cv.astype(np.float64)
+    state, conv = h.dev(st, torch.float32), h.dev(cv, ad)
+    dA, dD, dcw, dcb, dbias = (h.dev(a, torch.float32) for a in (A, D, cw, cb, bias))
+    for rd in range(3):
+        b = r.batch()
+        t = {n: h.dev(b[n], ad) for n in ("x", "z", "dt", "B", "C")}
+        y = torch.full(t["x"].shape, float("nan"), device="cuda", dtype=torch.float32)
+        ver.verify(state, conv, t["x"], t["dt"], t["B"], t["C"], dA, dD, dcw, dcb, t["z"], y, h.dev(b["n_prev"], torch.int32),
+                   s.k, dt_bias=dbias)
+        torch.cuda.synchronize()
+        assert ("stream" in ver.last_kernel) == (kernel == STREAM)
+        dt_eff = oracle.softplus_dt(np.nan_to_num(b["dt"]), bias)
+        fn = oracle.verify_m1 if m1 else oracle.verify
+        y_ref, o_state, o_conv = fn(o_state, o_conv, b["x"], dt_eff, b["B"], b["C"], A, D, cw, cb, b["z"], b["n_prev"], s.k,
+                                    s.flags, threads=oracle.host_threads())
+        yg = y.cpu().numpy().astype(np.float64)
+        valid = ~np.isnan(y_ref)
+        assert np.isnan(yg[~valid]).all() and not np.isnan(yg[valid]).any()
+        assert h.rel_l2(yg[valid], y_ref[valid]) <= 1e-5, f"round {rd}"
+        assert h.rel_l2(state.cpu().numpy(), o_state) <= 1e-5, f"round {rd}"
+        r.accept(synth.acceptance(s, rd))
+    assert ver.status() == 0
+    ver.close()
+
+
+@pytest.mark.parametrize("s,kernel", [(synth.CONFIGS[0], GENERIC), (synth.SWEEP[(4, 4)], STREAM), (synth.SWEEP[(4, 4)], GENERIC),
+                                      (synth.CONFIGS[3], STREAM)])
+def test_commit_selects_h_k_after_a_fully_accepted_round(s, kernel):
+    """Algorithm 2: a round whose drafts were all accepted keeps h_k, any other keeps h_j and replays.  Eight
+    rounds with a mix of full and partial acceptance through verify + commit on two buffers per sequence; the
+    returned rows and, at the end, each sequence's cache (wherever commit left it) against the oracle's plain
+    sequential run over the accepted tokens."""
+    h = H()
+    from paper_2408_15237_b200 import binding
+    flags = s.flags | binding.FLAG_STATE_K | binding.FLAG_COMMIT_SELECTS | binding.FLAG_Y_F32
+    ver = binding.Verifier(s.Bt, s.H, s.P, s.N, s.GB, s.GC, s.W, s.k, act=s.act, flags=flags, kernel=kernel)
+    ad = h.act_dtype(s)
+    A, D, cw, cb = synth.layer_params(s)
+    st, cv = synth.initial_cache(s)
+    rounds = 8
+    L = rounds * s.k + s.k + 1
+    stream = synth.token_stream(s, 0, L)
+    r = synth.Rounds(s, stream, first_j=0)
+    bufs = [(h.dev(st, torch.float32), h.dev(cv, ad)), (torch.full_like(h.dev(st, torch.float32), float("nan")),
+                                                        torch.zeros_like(h.dev(cv, ad)))]
+    dA, dD, dcw, dcb = (h.dev(a, torch.float32) for a in (A, D, cw, cb))
+    y_seq, st_seq, cv_seq = None, None, None
+    g = np.random.default_rng(7)
+    total = np.zeros(s.Bt, dtype=np.int64)
+    got_rows = {}
+    for rd in range(rounds):
+        b = r.batch()
+        t = {n: h.dev(b[n], ad) for n in ("x", "z", "dt", "B", "C")}
+        y = torch.full(t["x"].shape, float("nan"), device="cuda", dtype=torch.float32)
+        ver.verify(bufs[0][0], bufs[0][1], t["x"], t["dt"], t["B"], t["C"], dA, dD, dcw, dcb, t["z"], y, None, s.k,
+                   state_k=bufs[1][0], conv_state_k=bufs[1][1])
+        torch.cuda.synchronize()
+        assert ("stream" in ver.last_kernel) == (kernel == STREAM)
+        # the pending lengths the library used must be what this bookkeeping expects
+        assert ver_n_prev(ver, s.Bt) == [int(v) for v in b["n_prev"]]
+        yg = y.cpu().numpy().astype(np.float64)
+        rows = r.rows()
+        for bi in range(s.Bt):
+            for ti in range(rows.shape[1]):
+                if rows[bi, ti] >= 0:
+                    got_rows[(bi, int(rows[bi, ti]))] = yg[bi, ti]
+        # a mix: about half of the sequences accept everything, the others a random prefix
+        a = np.where(g.random(s.Bt) < 0.5, s.k, g.integers(0, s.k + 1, s.Bt)).astype(np.int32)
+        ver.commit(h.dev(a, torch.int32))
+        total += a
+        # the harness's bookkeeping of what is pending: nothing after a full acceptance
+        r.cursor = r.cursor + a
+        r.n_prev = np.where(a == s.k, 0, a).astype(np.int32)
+    torch.cuda.synchronize()
+    sel = ver.selection(s.Bt)
+    # a last flush folds what is still pending into the caches
+    b = r.batch(k=0)
+    t = {n: h.dev(np.nan_to_num(b[n]), ad) for n in ("x", "z", "dt", "B", "C")}
+    y = torch.full(t["x"].shape, float("nan"), device="cuda", dtype=torch.float32)
+    ver.verify(bufs[0][0], bufs[0][1], t["x"], t["dt"], t["B"], t["C"], dA, dD, dcw, dcb, t["z"], y, None, 0,
+               state_k=bufs[1][0], conv_state_k=bufs[1][1])
+    torch.cuda.synchronize()
+    assert ver.status() == 0
+    y_seq, st_seq, cv_seq = oracle.sequential(st, cv, stream["x"], stream["dt"], stream["B"], stream["C"], A, D, cw, cb,
+                                              stream["z"], total.astype(np.int32), s.flags, threads=oracle.host_threads())
+    for bi in range(s.Bt):
+        cur = bufs[sel[bi]]
+        assert h.rel_l2(cur[0][bi].cpu().numpy(), st_seq[bi]) <= 1e-5, f"sequence {bi}: cache"
+        assert np.abs(cur[1][bi].float().cpu().numpy().astype(np.float64) - cv_seq[bi]).max() == 0.0, f"sequence {bi}: window"
+    # every returned row of an accepted position equals the sequential run's row there
+    for (bi, pos), row in got_rows.items():
+        if pos < total[bi]:
+            assert h.rel_l2(row, y_seq[bi, pos]) <= 1e-5, (bi, pos)
+    ver.close()
+
+
+def ver_n_prev(ver, batch):
+    from paper_2408_15237_b200 import binding
+    return binding.mamba_spec_get_n_prev(ver.ctx, batch)
