@@ -164,6 +164,22 @@ int mamba_spec_verify(mamba_spec_ctx *ctx, void *state, void *conv_state, const 
  * holds h_k instead and has nothing pending (see the flag). */
 int mamba_spec_commit(mamba_spec_ctx *ctx, const int32_t *accept_len, int32_t batch, void *stream);
 
+/* The verification call for a caller that hands over only the k_draft NEW rows of every sequence (Sec. 4.2:
+ * "caching older entries"; Sec. 4.3, footnote: a circular buffer keeps old entries available for
+ * recomputation).  The context keeps, per layer, the rows of the last call: the tokens accepted since -- the
+ * first n_prev_accepted[b] of them, as recorded by mamba_spec_commit -- are replayed from there, so
+ *   x_new, io->z   [batch][k_draft][H][P]      dt_new  [batch][k_draft][H]  ([..][H*P] with FLAG_MAMBA1)
+ *   B_new          [batch][k_draft][G_B][N]    C_new   [batch][k_draft][G_C][N]
+ *   io->y          [batch][k_draft][H][P], output: the rows of the new tokens only (the replayed rows'
+ *                  outputs went out in the last call); io->t_max is ignored
+ * state, conv_state, A, D, io->conv_w/conv_b/state_k/conv_state_k/dt_bias as in mamba_spec_verify.
+ * One extra kernel lays the replayed and the new rows out for the verification kernel and keeps the new rows
+ * for the next call; the row store (n_layers x batch_max x k_max rows per tensor) is allocated on the first
+ * call.  The pending lengths are the context's (mamba_spec_commit); k_draft = 0 flushes them. */
+int mamba_spec_verify_new(mamba_spec_ctx *ctx, void *state, void *conv_state, const void *x_new, const void *dt_new,
+                          const void *B_new, const void *C_new, const float *A, const float *D, int32_t k_draft,
+                          const mamba_spec_io *io);
+
 /* Same computation with the per-step tensors in HOST memory (pinned memory
  * makes the copies asynchronous): x, dt, B, C, n_prev_accepted (nullable), io->z
  * are copied to context-owned device staging on io->stream, the kernel runs,

@@ -48,6 +48,8 @@ lib.mamba_spec_init.restype = ctypes.c_int
 lib.mamba_spec_init.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(_vp)]
 lib.mamba_spec_verify.restype = ctypes.c_int
 lib.mamba_spec_verify.argtypes = [_vp] * 10 + [_i32, ctypes.POINTER(IO)]
+lib.mamba_spec_verify_new.restype = ctypes.c_int
+lib.mamba_spec_verify_new.argtypes = [_vp] * 9 + [_i32, ctypes.POINTER(IO)]
 lib.mamba_spec_verify_host.restype = ctypes.c_int
 lib.mamba_spec_verify_host.argtypes = [_vp] * 10 + [_i32, ctypes.POINTER(IO)]
 lib.mamba_spec_verify_host_static.restype = ctypes.c_int
@@ -101,6 +103,11 @@ def _check(ctx, rc):
 def mamba_spec_verify(ctx, state, conv_state, x, dt, B, C, A, D, n_prev_accepted, k_draft, io: IO) -> None:
     _check(ctx, lib.mamba_spec_verify(ctx, _ptr(state), _ptr(conv_state), _ptr(x), _ptr(dt), _ptr(B), _ptr(C),
                                       _ptr(A), _ptr(D), _ptr(n_prev_accepted), int(k_draft), ctypes.byref(io)))
+
+
+def mamba_spec_verify_new(ctx, state, conv_state, x_new, dt_new, B_new, C_new, A, D, k_draft, io: IO) -> None:
+    _check(ctx, lib.mamba_spec_verify_new(ctx, _ptr(state), _ptr(conv_state), _ptr(x_new), _ptr(dt_new), _ptr(B_new), _ptr(C_new),
+                                          _ptr(A), _ptr(D), int(k_draft), ctypes.byref(io)))
 
 
 def mamba_spec_verify_host(ctx, state, conv_state, x, dt, B, C, A, D, n_prev_accepted, k_draft, io: IO) -> None:
@@ -223,6 +230,13 @@ class Verifier:
                     raise ValueError(f"{name}: want contiguous CUDA {dtype} {shape}")
         io = self._io(conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k, conv_state_k, dt_bias)
         mamba_spec_verify(self.ctx, state, conv_state, x, dt, B, C, A, D, n_prev, k, io)
+
+    def verify_new(self, state, conv_state, x_new, dt_new, B_new, C_new, A, D, conv_w, conv_b, z_new, y_new, k, layer=0,
+                   stream=None, state_k=None, conv_state_k=None, dt_bias=None):
+        """Only the k new rows of every sequence ([batch, k, ...]); replayed rows come from the library's row store."""
+        batch = y_new.shape[0]
+        io = self._io(conv_w, conv_b, z_new, y_new, batch, layer, 0, stream, state_k, conv_state_k, dt_bias)
+        mamba_spec_verify_new(self.ctx, state, conv_state, x_new, dt_new, B_new, C_new, A, D, k, io)
 
     def commit(self, accept_len, stream=None):
         if stream is None:

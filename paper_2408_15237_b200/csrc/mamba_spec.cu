@@ -40,6 +40,10 @@ struct mamba_spec_ctx {
     void *st_x = nullptr, *st_dt = nullptr, *st_B = nullptr, *st_C = nullptr, *st_z = nullptr, *st_y = nullptr;
     int32_t *st_n_prev = nullptr;
     bool staging_ready = false;
+    // row store of mamba_spec_verify_new: per tensor (x, z, dt, B, C) the last call's new rows of every layer
+    // [n_layers][batch_max][k_max][row], and one set of slabs [batch_max][2 k_max][row] that the kernels read
+    void *ring[5] = {nullptr, nullptr, nullptr, nullptr, nullptr}, *slab[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool ring_ready = false;
     cudaStream_t last_stream = nullptr;
     int32_t last_k = -1;
     int64_t launches = 0;
@@ -105,6 +109,26 @@ struct DeviceGuard {
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 size_t act_bytes(const mamba_spec_config &c) { return c.act_dtype == MAMBA_SPEC_DTYPE_BF16 ? 2 : 4; }
+
+// Lays out the token rows of one verify_new call for one tensor: slab[b][t] = the row kept from the last
+// call for t < j_b (a token accepted since), then the k new rows; the new rows are kept for the next call.
+// One thread per (sequence, piece of a row); U is the widest unit that divides a row.
+template <typename U>
+__global__ void assemble_rows_kernel(U *slab, U *ring, const U *fresh, const int32_t *n_prev, int batch, int k, int k_max,
+                                     int slab_rows, int units, int j_cap) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)batch * units) return;
+    const int b = (int)(i / units), u = (int)(i % units);
+    int j = n_prev[b];
+    j = j < 0 ? 0 : (j > j_cap ? j_cap : j);   // (the verification kernel clamps the same way and flags it)
+    U *srow = slab + (size_t)b * slab_rows * units + u, *rrow = ring + (size_t)b * k_max * units + u;
+    for (int t = 0; t < j; ++t) srow[(size_t)t * units] = rrow[(size_t)t * units];
+    for (int t = 0; t < k; ++t) {
+        const U v = fresh[((size_t)b * k + t) * units + u];
+        srow[(size_t)(j + t) * units] = v;
+        rrow[(size_t)t * units] = v;
+    }
+}
 
 // Algorithm 2's choice of the state to keep: with `sel` a fully accepted sequence takes the buffer that holds
 // the state after all tokens (h_k) and has nothing pending; every other sequence keeps h_j and replays.
@@ -318,6 +342,83 @@ int mamba_spec_commit(mamba_spec_ctx *ctx, const int32_t *accept_len, int32_t ba
     return MAMBA_SPEC_OK;
 }
 
+static cudaError_t assemble_rows(void *slab, void *ring, const void *fresh, const int32_t *n_prev, int batch, int k, int k_max,
+                                 int slab_rows, size_t row_bytes, int j_cap, cudaStream_t s) {
+    const int unit = row_bytes % 16 == 0 ? 16 : row_bytes % 4 == 0 ? 4 : 2;
+    const int units = (int)(row_bytes / unit);
+    const long long n = (long long)batch * units;
+    const unsigned blocks = (unsigned)((n + 255) / 256);
+    if (unit == 16)
+        assemble_rows_kernel<uint4><<<blocks, 256, 0, s>>>((uint4 *)slab, (uint4 *)ring, (const uint4 *)fresh, n_prev, batch, k, k_max, slab_rows, units, j_cap);
+    else if (unit == 4)
+        assemble_rows_kernel<uint32_t><<<blocks, 256, 0, s>>>((uint32_t *)slab, (uint32_t *)ring, (const uint32_t *)fresh, n_prev, batch, k, k_max, slab_rows, units, j_cap);
+    else
+        assemble_rows_kernel<uint16_t><<<blocks, 256, 0, s>>>((uint16_t *)slab, (uint16_t *)ring, (const uint16_t *)fresh, n_prev, batch, k, k_max, slab_rows, units, j_cap);
+    return cudaGetLastError();
+}
+
+int mamba_spec_verify_new(mamba_spec_ctx *ctx, void *state, void *conv_state, const void *x_new, const void *dt_new,
+                          const void *B_new, const void *C_new, const float *A, const float *D, int32_t k_draft,
+                          const mamba_spec_io *io) {
+    if (!ctx) return fail(nullptr, MAMBA_SPEC_ERR_NOT_INIT, "verify_new: ctx is null");
+    if (!io) return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "verify_new: io is null");
+    const mamba_spec_config &c = ctx->cfg;
+    if (k_draft < 0 || k_draft > c.k_max) return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "verify_new: k_draft %d outside 0..%d", k_draft, c.k_max);
+    if (io->batch < 1 || io->batch > c.batch_max) return fail(ctx, MAMBA_SPEC_ERR_BAD_SHAPE, "verify_new: batch %d outside 1..%d", io->batch, c.batch_max);
+    if (io->layer < 0 || io->layer >= c.n_layers) return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "verify_new: layer %d outside 0..%d", io->layer, c.n_layers - 1);
+    const bool gate = (c.flags & MAMBA_SPEC_FLAG_GATE) != 0;
+    if (k_draft > 0 && (!x_new || !dt_new || !B_new || !C_new || (gate && !io->z)))
+        return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "verify_new: a required tensor pointer is null");
+    if (c.k_max < 1) return fail(ctx, MAMBA_SPEC_ERR_UNSUPPORTED, "verify_new: the context was made with k_max = 0");
+    DeviceGuard guard(c.device);
+    if (!guard.ok) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "verify_new: cannot select device %d", c.device);
+    const size_t ab = act_bytes(c), hp = (size_t)c.n_heads * c.head_dim;
+    const size_t row_bytes[5] = {hp * ab, hp * ab, ((c.flags & MAMBA_SPEC_FLAG_MAMBA1) ? hp : (size_t)c.n_heads) * ab,
+                                 (size_t)c.n_groups_b * c.d_state * ab, (size_t)c.n_groups_c * c.d_state * ab};
+    const int slab_rows = 2 * c.k_max;
+    if (!ctx->ring_ready) {   // all or nothing
+        cudaError_t e = cudaSuccess;
+        for (int i = 0; i < 5 && e == cudaSuccess; ++i) {
+            // (16 spare bytes: the streaming kernel's boxes may read a little past the last row of dt)
+            e = cudaMalloc(&ctx->ring[i], (size_t)c.n_layers * c.batch_max * c.k_max * row_bytes[i] + 16);
+            if (e == cudaSuccess) e = cudaMalloc(&ctx->slab[i], (size_t)c.batch_max * slab_rows * row_bytes[i] + 16);
+            if (e == cudaSuccess) e = cudaMemset(ctx->slab[i], 0, (size_t)c.batch_max * slab_rows * row_bytes[i] + 16);
+            if (e == cudaSuccess) e = cudaMemset(ctx->ring[i], 0, (size_t)c.n_layers * c.batch_max * c.k_max * row_bytes[i] + 16);
+        }
+        if (e != cudaSuccess) {
+            for (int i = 0; i < 5; ++i) {
+                if (ctx->ring[i]) cudaFree(ctx->ring[i]);
+                if (ctx->slab[i]) cudaFree(ctx->slab[i]);
+                ctx->ring[i] = ctx->slab[i] = nullptr;
+            }
+            return fail(ctx, MAMBA_SPEC_ERR_CUDA, "verify_new: row store allocation failed: %s", cudaGetErrorString(e));
+        }
+        ctx->ring_ready = true;
+    }
+    cudaStream_t s = (cudaStream_t)io->stream;
+    const void *fresh[5] = {x_new, io->z, dt_new, B_new, C_new};
+    for (int i = 0; i < 5; ++i) {
+        if (i == 1 && !gate) continue;
+        char *ring = (char *)ctx->ring[i] + (size_t)io->layer * c.batch_max * c.k_max * row_bytes[i];
+        CUDA_TRY(ctx, assemble_rows(ctx->slab[i], ring, fresh[i], ctx->d_n_prev, io->batch, k_draft, c.k_max, slab_rows, row_bytes[i],
+                                    c.k_max, s));
+        ctx->launches++;
+    }
+    mamba_spec_io dio = *io;
+    dio.z = gate ? ctx->slab[1] : nullptr;
+    dio.t_max = slab_rows;
+    VerifyParams p;
+    int rc = check_and_fill(ctx, p, state, conv_state, ctx->slab[0], ctx->slab[2], ctx->slab[3], ctx->slab[4], A, D, nullptr, k_draft, &dio,
+                            "verify_new");
+    if (rc) return rc;
+    p.flags |= kFlagYNewOnly;
+    rc = launch(ctx, p, s, "verify_new");
+    if (rc) return rc;
+    ctx->last_stream = s;
+    ctx->last_k = k_draft;
+    return MAMBA_SPEC_OK;
+}
+
 int mamba_spec_verify_host(mamba_spec_ctx *ctx, void *state, void *conv_state, const void *x_host,
                            const void *dt_host, const void *B_host, const void *C_host, const float *A,
                            const float *D, const int32_t *n_prev_accepted_host, int32_t k_draft,
@@ -522,6 +623,10 @@ void mamba_spec_destroy(mamba_spec_ctx *ctx) {
         DeviceGuard guard(ctx->cfg.device);
         if (guard.ok) {
             cudaDeviceSynchronize();
+            for (int i = 0; i < 5; ++i) {
+                if (ctx->ring[i]) cudaFree(ctx->ring[i]);
+                if (ctx->slab[i]) cudaFree(ctx->slab[i]);
+            }
             void *bufs[] = {ctx->d_n_prev, ctx->d_status, ctx->d_sel, ctx->st_x, ctx->st_dt, ctx->st_B, ctx->st_C,
                             ctx->st_z, ctx->st_y, ctx->st_n_prev};
             for (void *b : bufs)

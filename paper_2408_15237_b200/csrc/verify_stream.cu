@@ -664,7 +664,9 @@ __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const Stream
     {
         const float *xcs = reinterpret_cast<const float *>(gb + L.c_xc), *gz = reinterpret_cast<const float *>(gb + L.c_gz);
         const float *Gm = reinterpret_cast<const float *>(gb + L.c_G);
-        const size_t y0 = (((size_t)b * p.t_max) * p.H + h) * p.P + rc * CR;
+        // (with new rows only, y is [batch][k]: token j is its row 0 and the replayed rows' outputs are dropped)
+        const bool y_new = (p.flags & kFlagYNewOnly) != 0;
+        const size_t y0 = (((size_t)b * (y_new ? p.k : p.t_max) - (y_new ? j : 0)) * p.H + h) * p.P + rc * CR;
         const size_t tstride = (size_t)p.H * p.P;
         // a thread's elements share their row (the group's thread count is a multiple of CR): its xc values
         // are read once; D sits on the diagonal of G
@@ -693,6 +695,7 @@ __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const Stream
             float y = fmaf(hc->alpha[t], v, w);
             if (gate) y *= gz[e];
             const size_t yi = y0 + t * tstride + row;
+            if (y_new && t < j) continue;
             if (y_f32) reinterpret_cast<float *>(p.y)[yi] = y;
             else reinterpret_cast<__nv_bfloat16 *>(p.y)[yi] = __float2bfloat16_rn(y);
         }
@@ -933,7 +936,6 @@ StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, si
     };
     if (!bf16) return reject("activations are not bf16");
     if (p.flags & kFlagMamba1) return reject("the Mamba-1 parameterisation runs in the generic kernel");
-    if (p.flags & kFlagYNewOnly) return reject("variant not in the streaming kernel");
     if (p.W != kW) return reject("conv width is not 4");
     if (p.N != 64 && p.N != 128) return reject("state dim is not 64 or 128");
     if (p.P % 32) return reject("head dim is not a multiple of 32");

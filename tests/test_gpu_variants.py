@@ -182,3 +182,73 @@ def test_commit_selects_h_k_after_a_fully_accepted_round(s, kernel):
 def ver_n_prev(ver, batch):
     from paper_2408_15237_b200 import binding
     return binding.mamba_spec_get_n_prev(ver.ctx, batch)
+
+
+@pytest.mark.parametrize("s,kernel,selects", [(synth.CONFIGS[0], GENERIC, False), (synth.SWEEP[(4, 4)], STREAM, False),
+                                              (synth.SWEEP[(4, 4)], STREAM, True), (synth.SWEEP[(4, 4)], GENERIC, True),
+                                              (synth.CONFIGS[3], STREAM, True)])
+def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects):
+    """The caller hands over only the k new rows per round (Sec. 4.2 "caching older entries"); the tokens accepted
+    since the last call are replayed from the rows the library kept.  Two layers share the context (each has
+    its own kept rows).  Mixed full and partial acceptance over eight rounds; returned rows, final caches and
+    conv windows against the oracle's plain sequential run."""
+    h = H()
+    from paper_2408_15237_b200 import binding
+    n_layers = 2
+    flags = s.flags | binding.FLAG_Y_F32 | ((binding.FLAG_STATE_K | binding.FLAG_COMMIT_SELECTS) if selects else 0)
+    ver = binding.Verifier(s.Bt, s.H, s.P, s.N, s.GB, s.GC, s.W, s.k, act=s.act, flags=flags, kernel=kernel, n_layers=n_layers)
+    ad = h.act_dtype(s)
+    rounds = 8
+    L = rounds * s.k + 1
+    lay = []
+    for l in range(n_layers):
+        A, D, cw, cb = synth.layer_params(s, l)
+        st, cv = synth.initial_cache(s, l)
+        stream = synth.token_stream(s, l, L)
+        bufs = [(h.dev(st, torch.float32), h.dev(cv, ad)),
+                (torch.full_like(h.dev(st, torch.float32), float("nan")), torch.zeros_like(h.dev(cv, ad)))]
+        lay.append(dict(np=(A, D, cw, cb, st, cv), stream=stream, bufs=bufs, got={},
+                        dev=tuple(h.dev(a, torch.float32) for a in (A, D, cw, cb))))
+    g = np.random.default_rng(11)
+    cursor = np.zeros(s.Bt, dtype=np.int64)     # tokens verified so far
+    for rd in range(rounds):
+        for l, q in enumerate(lay):
+            idx = cursor[:, None] + np.arange(s.k)[None, :]
+            bi = np.arange(s.Bt)[:, None]
+            t = {n: h.dev(q["stream"][n][bi, idx], ad) for n in ("x", "z", "dt", "B", "C")}
+            y = torch.full((s.Bt, s.k, s.H, s.P), float("nan"), device="cuda", dtype=torch.float32)
+            dA, dD, dcw, dcb = q["dev"]
+            ver.verify_new(q["bufs"][0][0], q["bufs"][0][1], t["x"], t["dt"], t["B"], t["C"], dA, dD, dcw, dcb, t["z"], y, s.k,
+                           layer=l, state_k=q["bufs"][1][0] if selects else None, conv_state_k=q["bufs"][1][1] if selects else None)
+            torch.cuda.synchronize()
+            assert ("stream" in ver.last_kernel) == (kernel == STREAM)
+            yg = y.cpu().numpy().astype(np.float64)
+            for b in range(s.Bt):
+                for i in range(s.k):
+                    q["got"][(b, int(cursor[b] + i))] = yg[b, i]
+        a = np.where(g.random(s.Bt) < 0.4, s.k, g.integers(0, s.k + 1, s.Bt)).astype(np.int32)
+        ver.commit(h.dev(a, torch.int32))
+        cursor += a
+    # flush what is pending
+    for l, q in enumerate(lay):
+        dA, dD, dcw, dcb = q["dev"]
+        y = torch.zeros((s.Bt, 1, s.H, s.P), device="cuda", dtype=torch.float32)
+        ver.verify_new(q["bufs"][0][0], q["bufs"][0][1], None, None, None, None, dA, dD, dcw, dcb, None, y, 0, layer=l,
+                       state_k=q["bufs"][1][0] if selects else None, conv_state_k=q["bufs"][1][1] if selects else None)
+    torch.cuda.synchronize()
+    assert ver.status() == 0
+    sel = ver.selection(s.Bt) if selects else [0] * s.Bt
+    for l, q in enumerate(lay):
+        A, D, cw, cb, st, cv = q["np"]
+        y_seq, st_seq, cv_seq = oracle.sequential(st, cv, q["stream"]["x"], q["stream"]["dt"], q["stream"]["B"], q["stream"]["C"],
+                                                  A, D, cw, cb, q["stream"]["z"], cursor.astype(np.int32), s.flags,
+                                                  threads=oracle.host_threads())
+        for b in range(s.Bt):
+            cur = q["bufs"][sel[b]]
+            assert h.rel_l2(cur[0][b].cpu().numpy(), st_seq[b]) <= 1e-5, f"layer {l} sequence {b}: cache"
+            assert np.abs(cur[1][b].float().cpu().numpy().astype(np.float64) - cv_seq[b]).max() == 0.0
+        for (b, pos), row in q["got"].items():
+            if pos < cursor[b]:
+                assert not np.isnan(row).any()
+                assert h.rel_l2(row, y_seq[b, pos]) <= 1e-5, (l, b, pos)
+    ver.close()
