@@ -233,6 +233,13 @@ int mamba_spec_get_n_prev(mamba_spec_ctx *ctx, int32_t *n_prev_host, int32_t bat
  * shares the context, since all layers see the same commits.  Synchronises. */
 int mamba_spec_get_selection(mamba_spec_ctx *ctx, int32_t *sel_host, int32_t batch);
 
+/* Which kernel a verify call of this shape would run, and with which launch plan, as text in buf (HOST,
+ * buf_len bytes): "stream<...>" with the streaming kernel's ring depths, groups and grid, or "generic (reason)".
+ * Host logic only: no tensor is touched and no kernel launched.  sm_count / smem_per_block describe the GPU
+ * (multiprocessors, opt-in shared memory per block in bytes); pass 0 for both to ask the CUDA device cfg names. */
+int mamba_spec_describe_plan(const mamba_spec_config *cfg, int32_t batch, int32_t t_max, int32_t k_draft,
+                             int32_t sm_count, int64_t smem_per_block, char *buf, int32_t buf_len);
+
 /* Number of kernels this context has launched so far (HOST counter). */
 int64_t mamba_spec_launch_count(const mamba_spec_ctx *ctx);
 

@@ -62,6 +62,8 @@ lib.mamba_spec_get_n_prev.restype = ctypes.c_int
 lib.mamba_spec_get_n_prev.argtypes = [_vp, ctypes.POINTER(_i32), _i32]
 lib.mamba_spec_get_selection.restype = ctypes.c_int
 lib.mamba_spec_get_selection.argtypes = [_vp, ctypes.POINTER(_i32), _i32]
+lib.mamba_spec_describe_plan.restype = ctypes.c_int
+lib.mamba_spec_describe_plan.argtypes = [ctypes.POINTER(Config), _i32, _i32, _i32, _i32, ctypes.c_int64, ctypes.c_char_p, _i32]
 lib.mamba_spec_launch_count.restype = ctypes.c_int64
 lib.mamba_spec_launch_count.argtypes = [_vp]
 lib.mamba_spec_last_kernel.restype = ctypes.c_char_p
@@ -146,6 +148,15 @@ def mamba_spec_get_selection(ctx, batch):
     buf = (_i32 * batch)()
     _check(ctx, lib.mamba_spec_get_selection(ctx, buf, batch))
     return list(buf)
+
+
+def mamba_spec_describe_plan(cfg: Config, batch, t_max, k_draft, sm_count=0, smem_per_block=0) -> str:
+    """Which kernel and launch plan a call of this shape gets (host logic only)."""
+    buf = ctypes.create_string_buffer(256)
+    rc = lib.mamba_spec_describe_plan(ctypes.byref(cfg), batch, t_max, k_draft, sm_count, smem_per_block, buf, 256)
+    if rc != OK:
+        raise MambaSpecError(rc, lib.mamba_spec_last_error(None).decode())
+    return buf.value.decode()
 
 
 def mamba_spec_launch_count(ctx) -> int:

@@ -27,38 +27,48 @@ def _nvcc() -> str:
     return exe
 
 
-def _stale() -> bool:
-    if not LIB.exists():
+def _stale(lib: Path = LIB) -> bool:
+    if not lib.exists():
         return True
     deps = list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "mamba_spec.h"]
-    return any(d.stat().st_mtime > LIB.stat().st_mtime for d in deps)
+    return any(d.stat().st_mtime > lib.stat().st_mtime for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> Path:
-    if not force and not _stale():
-        return LIB
+# Test-only build: the same sources with waits that give up after about a millisecond and a barrier that can
+# never complete, so that the kernel's give-up path runs (every copy still lands; see tests/test_gpu_waits.py).
+WAIT_TEST_LIB = PKG / "_build" / "libmamba_spec_waittest.so"
+WAIT_TEST_DEFINES = ["-DMSPEC_WAIT_LIMIT_CYCLES=2000000ll", "-DMSPEC_TEST_RAW_NEVER_FULL=1"]
+
+
+def build_wait_test_library(force: bool = False) -> Path:
+    return build_library(force=force, defines=WAIT_TEST_DEFINES, out=WAIT_TEST_LIB, tag="waittest")
+
+
+def build_library(force: bool = False, verbose: bool = False, defines=(), out: Path = LIB, tag: str = "") -> Path:
+    if not force and not _stale(out):
+        return out
     objs = []
     out_dir = PKG / "_build"
     out_dir.mkdir(exist_ok=True)
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = (["-Xptxas", "-v"] if verbose else []) + list(defines)
     procs = []
     for src in SOURCES:
-        obj = out_dir / (src + ".o")
+        obj = out_dir / (src + (f".{tag}" if tag else "") + ".o")
         cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", str(CSRC / src), "-o", str(obj)]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     for src, pr in procs:
-        out, _ = pr.communicate()
+        log, _ = pr.communicate()
         if verbose or pr.returncode:
-            sys.stderr.write(out)
+            sys.stderr.write(log)
         if pr.returncode:
             raise RuntimeError(f"nvcc failed on {src}")
-    tmp = PKG / f".libmamba_spec.{os.getpid()}.so"
+    tmp = out.parent / f".{out.stem}.{os.getpid()}.so"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", str(tmp), *map(str, objs),
            "-lcudart"]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":

@@ -611,6 +611,40 @@ int mamba_spec_get_selection(mamba_spec_ctx *ctx, int32_t *sel_host, int32_t bat
     return MAMBA_SPEC_OK;
 }
 
+int mamba_spec_describe_plan(const mamba_spec_config *cfg, int32_t batch, int32_t t_max, int32_t k_draft,
+                             int32_t sm_count, int64_t smem_per_block, char *buf, int32_t buf_len) {
+    if (!cfg || !buf || buf_len < 1) return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "describe_plan: null cfg or buffer");
+    const mamba_spec_config &c = *cfg;
+    if (c.n_heads < 1 || c.head_dim < 1 || c.d_state < 1 || c.n_groups_b < 1 || c.n_groups_c < 1 || c.n_heads % c.n_groups_b ||
+        c.n_heads % c.n_groups_c || batch < 1 || t_max < 1 || k_draft < 0 || k_draft > t_max || c.k_max < 0)
+        return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "describe_plan: shape out of range");
+    if (sm_count <= 0 || smem_per_block <= 0) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess)
+            return fail(nullptr, MAMBA_SPEC_ERR_CUDA, "describe_plan: no CUDA device %d to ask", c.device);
+        sm_count = prop.multiProcessorCount;
+        smem_per_block = (int64_t)prop.sharedMemPerBlockOptin;
+    }
+    VerifyParams p;
+    memset(&p, 0, sizeof p);
+    p.batch = batch; p.t_max = t_max; p.H = c.n_heads; p.P = c.head_dim; p.N = c.d_state;
+    p.GB = c.n_groups_b; p.GC = c.n_groups_c; p.W = c.conv_width; p.k = k_draft;
+    p.j_cap = c.k_max < t_max - k_draft ? c.k_max : t_max - k_draft;
+    p.flags = c.flags;
+    // the planner only looks at whether these are set
+    p.z = (c.flags & MAMBA_SPEC_FLAG_GATE) ? (const void *)buf : nullptr;
+    p.state_k = (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? (float *)buf : nullptr;
+    const bool bf16 = c.act_dtype == MAMBA_SPEC_DTYPE_BF16;
+    if (c.kernel_select != MAMBA_SPEC_KERNEL_GENERIC) {
+        const StreamPlan plan = plan_verify_stream(p, bf16, sm_count, (size_t)smem_per_block);
+        if (plan.ok) snprintf(buf, (size_t)buf_len, "%s", plan.name);
+        else snprintf(buf, (size_t)buf_len, "generic (%s)", plan.name);
+    } else {
+        snprintf(buf, (size_t)buf_len, "generic (selected)");
+    }
+    return MAMBA_SPEC_OK;
+}
+
 int64_t mamba_spec_launch_count(const mamba_spec_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 const char *mamba_spec_last_kernel(const mamba_spec_ctx *ctx) { return ctx ? ctx->last_kernel : "none"; }

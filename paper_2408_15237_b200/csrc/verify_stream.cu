@@ -76,6 +76,7 @@ struct Ctrl {
     unsigned long long raw_full[kMaxR], raw_empty[kMaxR];
     int abort;
     int state_par[kMaxS];  // parity of the producer's last fill of each state stage, -1 before any
+    int raw_par[kMaxR];    // the same for the raw stages
     int jarr[kJTable];
     float A[kMaxHeads], D[kMaxHeads];
     int walk[1 + 8 + 4 * kGroups];   // a WalkInfo, see below
@@ -251,7 +252,13 @@ __device__ __forceinline__ bool issue_raw(const VerifyParams &p, const StreamLay
     if (!mbar_wait(smem_u32(&ctl.raw_empty[rs]), (uint32_t)rp ^ 1u, &ctl.abort)) return false;
     const uint32_t raw = smem_base + L.raw_off + rs * L.raw_stride, bar = smem_u32(&ctl.raw_full[rs]);
     const int c0 = h * p.P + rc * CR, row0 = b * p.t_max;
-    if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)L.raw_tx);
+#ifdef MSPEC_TEST_RAW_NEVER_FULL
+    // Test build only: one transaction byte more is expected than is requested, so every copy lands and the
+    // barrier still never completes -- the consumers' bounded wait runs out.
+    if (lane == 0) { ctl.raw_par[rs] = rp; mbar_arrive_expect_tx(bar, (uint32_t)L.raw_tx + 16u); }
+#else
+    if (lane == 0) { ctl.raw_par[rs] = rp; mbar_arrive_expect_tx(bar, (uint32_t)L.raw_tx); }
+#endif
     __syncwarp();
     // One tensor-load instruction for the six 2-D boxes (lane l takes map l of InputMaps: x, z, B, C, dt,
     // conv window) and one bulk-copy instruction for taps and bias: issued convergently, the requests queue
@@ -787,6 +794,7 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
             mbar_init(smem_u32(&ctl.raw_empty[s]), kGroupWarps);
         }
         for (int s = 0; s < kMaxS; ++s) ctl.state_par[s] = -1;
+        for (int s = 0; s < kMaxR; ++s) ctl.raw_par[s] = -1;
         ctl.abort = 0;
         fence_mbar_init();
         WalkInfo &wi = *reinterpret_cast<WalkInfo *>(ctl.walk);
@@ -854,6 +862,12 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
             const long long t0 = clock64();
             if (ctl.state_par[s] >= 0)
                 while (!mbar_try_park(smem_u32(&ctl.state_full[s]), (uint32_t)ctl.state_par[s], 20000u) &&
+                       clock64() - t0 < kWaitLimitCycles) {}
+        }
+        for (int s = 0; s < L.R; ++s) {
+            const long long t0 = clock64();
+            if (ctl.raw_par[s] >= 0)
+                while (!mbar_try_park(smem_u32(&ctl.raw_full[s]), (uint32_t)ctl.raw_par[s], 20000u) &&
                        clock64() - t0 < kWaitLimitCycles) {}
         }
     }
@@ -1010,6 +1024,10 @@ StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, si
     // with few chunks per CTA the state requests should not queue behind a second chunk's small inputs
     // (measured: batch 4 and 16 gain 2 % with lead 0, batch 64 loses 1 %)
     if (per_cta <= 16) L.lead = 0;
+    // A group hands a stage with a pending store back only when it starts its next chunk, after that chunk's
+    // small inputs are in; the producer requests those only once it has the stage (lead 0), or one chunk earlier
+    // (lead 1).  So no more groups than stages + lead may hold stages, unless the CTA never reuses a stage.
+    while (L.ngroups > 1 && L.ngroups > S + L.lead && per_cta > S) --L.ngroups;
     L.S = S;
     L.state_off = (kCtrlBytes + 1023) & ~1023;   // the swizzled state stages need 1024-byte alignment
     L.raw_off = L.state_off + S * L.state_stride;

@@ -310,3 +310,55 @@ def test_second_snapshot_after_all_tokens(s, kernel):
     assert ("stream" in ver.last_kernel) == (kernel == STREAM)
     assert ver.status() == 0
     ver.close()
+
+
+@pytest.mark.parametrize("kernel", [GENERIC, STREAM])
+def test_checkpoint_and_resume_in_a_fresh_context(kernel):
+    """A decoder's whole resumable state per layer is the cached state, the conv window and the pending lengths
+    (Sec. 4.2; Sec. 4.3, footnote).  After round 3 these are saved, the context is destroyed, a fresh context
+    and fresh device buffers are loaded from the copy, and rounds 4..7 must come out bit for bit as in the run
+    that was never interrupted."""
+    h = H()
+    from paper_2408_15237_b200 import binding
+    s = synth.SWEEP[(4, 4)]
+    ad = h.act_dtype(s)
+    stream = synth.token_stream(s, 0, 8 * s.k + s.k + 1)
+    acc = [synth.acceptance(s, rd) for rd in range(8)]
+
+    def run(ver, lay, r, rounds):
+        outs = []
+        for rd in rounds:
+            b = r.batch()
+            t = {n: h.dev(b[n], ad) for n in ("x", "z", "dt", "B", "C")}
+            y = torch.full(t["x"].shape, float("nan"), device="cuda", dtype=ad)
+            ver.verify(lay.state, lay.conv, t["x"], t["dt"], t["B"], t["C"], lay.A, lay.D, lay.cw, lay.cb, t["z"], y, None, s.k)
+            ver.commit(h.dev(acc[rd], torch.int32))
+            torch.cuda.synchronize()
+            outs.append(y.clone())
+            r.accept(acc[rd])
+        return outs
+
+    # the uninterrupted run
+    ver_a, lay_a, r_a = h.make_verifier(s, kernel), h.Layer(s), synth.Rounds(s, stream)
+    run(ver_a, lay_a, r_a, range(4))
+    saved = dict(state=lay_a.state.cpu().clone(), conv=lay_a.conv.cpu().clone(), n_prev=binding.mamba_spec_get_n_prev(ver_a.ctx, s.Bt),
+                 cursor=r_a.cursor.copy())
+    want = run(ver_a, lay_a, r_a, range(4, 8))
+    want_state, want_conv = lay_a.state.clone(), lay_a.conv.clone()
+    ver_a.close()
+    # the resumed run: fresh context, fresh buffers, pending lengths handed back through commit
+    ver_b, lay_b, r_b = h.make_verifier(s, kernel), h.Layer(s), synth.Rounds(s, stream)
+    lay_b.state.copy_(saved["state"])
+    lay_b.conv.copy_(saved["conv"])
+    assert saved["n_prev"] == [int(v) for v in acc[3]]
+    # (a fresh context has no pending lengths yet: the saved ones go back in through commit, which clamps to the
+    #  draft length of the last verify, or to k_max when there has been none)
+    binding.lib.mamba_spec_commit(ver_b.ctx, h.dev(np.asarray(saved["n_prev"], dtype=np.int32), torch.int32).data_ptr(), s.Bt,
+                                  torch.cuda.current_stream().cuda_stream)
+    r_b.cursor, r_b.n_prev = saved["cursor"].copy(), np.asarray(saved["n_prev"], dtype=np.int32)
+    got = run(ver_b, lay_b, r_b, range(4, 8))
+    for a, b_ in zip(want, got):
+        assert torch.equal(torch.nan_to_num(a.float(), nan=-7.0), torch.nan_to_num(b_.float(), nan=-7.0))
+    assert torch.equal(lay_b.state, want_state) and torch.equal(lay_b.conv, want_conv)
+    assert ver_b.status() == 0
+    ver_b.close()
