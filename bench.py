@@ -34,9 +34,38 @@ from paper_2408_15237_b200 import synth  # noqa: E402
 METRIC = "verified_draft_tokens_per_s_per_mamba_layer"
 UNIT = "tokens/s/layer"
 N_ROUND_SETS = 8
-# dram__bytes_read.sum + dram__bytes_write.sum of one verify_stream_kernel<128,64> launch of this shape (ncu, 4-layer
-# capture, see profiles/verify_stream_config4_b16.md); None whenever the kernel has changed since it was taken.
-NCU_DRAM_BYTES_PER_LAUNCH = 37.49e6
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "verify_stream_dram_traffic.txt")
+KERNEL_SOURCES = ("paper_2408_15237_b200/csrc/verify_stream.cu", "paper_2408_15237_b200/csrc/common.cuh")
+
+
+def kernel_source_hash():
+    import hashlib
+    hsh = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            hsh.update(f.read())
+    return hsh.hexdigest()[:16]
+
+
+def measured_traffic(plan_name):
+    """DRAM bytes per launch of the streaming kernel from the kept ncu summary, or None when that summary was taken
+    with another plan or another version of the kernel's source (then it says nothing about this run)."""
+    rec = {}
+    try:
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                if "=" in line and not line.lstrip().startswith("#"):
+                    k, v = line.split("=", 1)
+                    rec[k.strip()] = v.strip()
+    except OSError:
+        return None, None
+    if rec.get("source_sha256_16") != kernel_source_hash() or rec.get("plan") != plan_name:
+        return None, None
+    try:
+        rd, wr = float(rec["dram_bytes_read_per_launch"]), float(rec["dram_bytes_write_per_launch"])
+    except (KeyError, ValueError):
+        return None, None
+    return rd + wr, {"dram_bytes_read": rd, "dram_bytes_write": wr, "capture": rec.get("capture", "")}
 
 
 def measured_peaks():
@@ -278,8 +307,10 @@ def isolated_launch_ms(stack, reps=5):
     return float(np.median([a.elapsed_time(b) for a, b in times]))
 
 
-def cpu_oracle_sample(s, calls, threads):
-    """Times the fp64 oracle, as it stands, on `calls` verify calls of one layer of the workload."""
+def cpu_oracle_sample(s, calls, threads, gpu_check=None):
+    """Times the fp64 oracle, as it stands, on `calls` verify calls of one layer of the workload.  `gpu_check`, if
+    given, gets the inputs and the oracle's results of the untimed first call (a parity spot check of the library
+    on the workload's own shape, outside every timed region)."""
     import oracle
     A, D, cw, cb = synth.layer_params(s, 0)
     st, cv = synth.initial_cache(s, 0)
@@ -287,8 +318,10 @@ def cpu_oracle_sample(s, calls, threads):
     r = synth.Rounds(s, stream, wrap=True)
     r.accept(synth.acceptance(s, 0))
     b = r.batch()      # one untimed call: compiles/loads the C library and touches the buffers
-    oracle.verify(st, cv, b["x"], b["dt"], b["B"], b["C"], A, D, cw, cb, b["z"], b["n_prev"], s.k, s.flags,
-                  threads=threads)
+    ref = oracle.verify(st, cv, b["x"], b["dt"], b["B"], b["C"], A, D, cw, cb, b["z"], b["n_prev"], s.k, s.flags,
+                        threads=threads)
+    if gpu_check is not None:
+        gpu_check(dict(A=A, D=D, cw=cw, cb=cb, state=st, conv=cv, batch=b), ref)
     per_call = []
     for c in range(calls):
         b = r.batch()
@@ -298,6 +331,33 @@ def cpu_oracle_sample(s, calls, threads):
         per_call.append(time.perf_counter() - t0)
         r.accept(synth.acceptance(s, c + 1))
     return per_call
+
+
+def parity_spot_check(s, out):
+    """Returns a callback for cpu_oracle_sample: runs the library on the same inputs and records the relative L2
+    errors of y (against the oracle rounded to the output precision and unrounded) and of the committed state."""
+    def check(inp, ref):
+        from paper_2408_15237_b200 import binding
+        y_ref, st_ref, _ = ref
+        ad = torch.bfloat16 if s.act == "bf16" else torch.float32
+        dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(device="cuda", dtype=dt)
+        ver = binding.Verifier(s.Bt, s.H, s.P, s.N, s.GB, s.GC, s.W, s.k, act=s.act, flags=s.flags)
+        b = inp["batch"]
+        t = {n: dev(np.nan_to_num(b[n]), ad) for n in ("x", "z", "dt", "B", "C")}
+        y = torch.zeros(t["x"].shape, device="cuda", dtype=ad)
+        state, conv = dev(inp["state"], torch.float32), dev(inp["conv"], ad)
+        ver.verify(state, conv, t["x"], t["dt"], t["B"], t["C"], dev(inp["A"], torch.float32), dev(inp["D"], torch.float32),
+                   dev(inp["cw"], torch.float32), dev(inp["cb"], torch.float32), t["z"], y, dev(b["n_prev"], torch.int32), s.k)
+        torch.cuda.synchronize()
+        valid = ~np.isnan(y_ref)
+        yg = y.float().cpu().numpy().astype(np.float64)
+        rel = lambda a, w: float(np.linalg.norm(a - w) / np.linalg.norm(w))
+        yq = synth.round_bf16(np.nan_to_num(y_ref).astype(np.float32)).astype(np.float64) if s.act == "bf16" else y_ref
+        out.update({"kernel": ver.last_kernel, "y_rel_l2_vs_unrounded_oracle": rel(yg[valid], y_ref[valid]),
+                    "y_rel_l2_vs_oracle_rounded_to_output_dtype": rel(yg[valid], yq[valid]),
+                    "state_rel_l2": rel(state.cpu().numpy().astype(np.float64), st_ref), "device_status": ver.status()})
+        ver.close()
+    return check
 
 
 def run_reference(args, s, rank):
@@ -429,6 +489,16 @@ def main():
         torch.cuda.synchronize()
         print(f"profile run: {stack.ver.launches} launches, kernel {stack.ver.last_kernel}, status {stack.ver.status()}")
         return
+    if args.gpus > 1 and "RANK" not in os.environ and not (args.sweep or args.multistep or args.draft):
+        # started plainly with --gpus N: become N ranks, one per GPU (replicas: the path does not shard)
+        import socket
+        import subprocess
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+               "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -480,16 +550,17 @@ def main():
     ms_e2e = max_over_ranks(ms_e2e, "cuda")
     e2e_value = job_value(world, s.Bt, s.k, s.n_layers, ms_e2e / e2e_steps)
 
-    cpu = None
+    cpu, spot = None, {}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         threads = oracle.host_threads()
-        calls = cpu_oracle_sample(s, 12, threads)
+        calls = cpu_oracle_sample(s, 12, threads, gpu_check=parity_spot_check(s, spot))
         sec = float(np.mean(calls[2:]))
         cpu = {"value": s.Bt * s.k / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"10 verify calls of one layer of the workload (batch {s.Bt}, k={s.k}), fp64, "
                          f"{threads} OpenMP threads over (sequence, head); {sec * 1e3:.1f} ms per call"}
 
+    traffic, traffic_detail = measured_traffic(stack.ver.last_kernel)
     if rank == 0:
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -500,7 +571,8 @@ def main():
                        "replicas": "each GPU runs the whole workload (no sharding, no collective)" if world > 1 else "single GPU",
                        "kernel": stack.ver.last_kernel, "device_status": status},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_DRAM_BYTES_PER_LAUNCH, "peak_source": peak_src, "algorithmic_bytes_per_launch": bytes_launch,
+                         "traffic": traffic, "traffic_detail": traffic_detail, "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": bytes_launch,
                          "us_per_launch": us_launch, "us_per_launch_isolated": iso_ms * 1e3,
                          "achieved_isolated": bytes_launch / (iso_ms * 1e-3) / 1e9, "frac_of_8TBps": achieved / 8000.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": host.h2d, "d2h_bytes_per_step": host.d2h,
@@ -510,6 +582,8 @@ def main():
         }
         if cpu:
             out["cpu_baseline"] = cpu
+        if spot:
+            out["parity_spot_check"] = spot
         print(json.dumps(out))
     stack.ver.close()
     if use_dist:

@@ -26,6 +26,11 @@ struct VerifyParams {
     const float *D;          // [H]; Mamba-1 form: [H*P]
     const float *dt_bias;    // [H] ([H*P] in the Mamba-1 form) or null: added to the raw interval before its softplus
     const int32_t *sel;      // [batch] or null: which of (state, state_k) holds each sequence's cache (commit-selects mode)
+    const int32_t *row_off;  // [batch] or null: token t of sequence b is row row_off[b] + row_off_const + t of its slab
+    int32_t row_off_const;   //   (later segments of a token block that is split over several launches)
+    int32_t row_off_cap;     //   largest legal row_off[b]
+    int32_t n_prev_done;     // pending rows of each sequence that earlier launches of this call have replayed already
+    int32_t n_prev_full;     //   and, when non-zero, the bound on n_prev[b] itself (j_cap bounds what is left of it)
     const float *conv_w;     // [H*P][W]
     const float *conv_b;     // [H*P]
     const int32_t *n_prev;   // [batch]
@@ -57,14 +62,27 @@ __device__ __forceinline__ float ld_act(const __nv_bfloat16 *p, size_t i) { retu
 __device__ __forceinline__ void st_act(float *p, size_t i, float v) { p[i] = v; }
 __device__ __forceinline__ void st_act(__nv_bfloat16 *p, size_t i, float v) { p[i] = __float2bfloat16_rn(v); }
 
+// First slab row of sequence b's tokens in this launch (0 unless the block was split; the offsets are pending
+// lengths, clamped like them).
+__device__ __forceinline__ int first_row(const VerifyParams &p, int b) {
+    int off = p.row_off_const;
+    if (p.row_off != nullptr) {
+        const int v = p.row_off[b];
+        off += v < 0 ? 0 : (v > p.row_off_cap ? p.row_off_cap : v);
+    }
+    return off;
+}
+
 // Reads n_prev[b], clamps it into [0, j_cap] and flags the status word if it had to.
 __device__ __forceinline__ int load_n_prev(const VerifyParams &p, int b) {
     int j = p.n_prev[b];
-    if (j < 0 || j > p.j_cap) {
+    const int full = p.n_prev_full ? p.n_prev_full : p.j_cap;
+    if (j < 0 || j > full) {
         atomicOr(p.status, kStatusNprevClamped);
-        j = j < 0 ? 0 : p.j_cap;
+        j = j < 0 ? 0 : full;
     }
-    return j;
+    j -= p.n_prev_done;
+    return j < 0 ? 0 : (j > p.j_cap ? p.j_cap : j);
 }
 
 // Launchers (defined in verify_generic.cu / verify_stream.cu).  Return cudaGetLastError().

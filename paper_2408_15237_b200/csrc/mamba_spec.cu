@@ -44,6 +44,11 @@ struct mamba_spec_ctx {
     // [n_layers][batch_max][k_max][row], and one set of slabs [batch_max][2 k_max][row] that the kernels read
     void *ring[5] = {nullptr, nullptr, nullptr, nullptr, nullptr}, *slab[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     bool ring_ready = false;
+    // token blocks of more than 16 rows go through the streaming kernel in segments: the state between two
+    // segments lives here (two of each, used in turn), plus a vector of zeros (nothing pending after the first)
+    float *split_state[2] = {nullptr, nullptr};
+    void *split_conv[2] = {nullptr, nullptr};
+    int32_t *d_zero = nullptr;
     cudaStream_t last_stream = nullptr;
     int32_t last_k = -1;
     int64_t launches = 0;
@@ -249,6 +254,7 @@ static int check_and_fill(mamba_spec_ctx *ctx, VerifyParams &p, void *state, voi
     p.conv_state = conv_state;
     p.x = x; p.dt = dt; p.B = B; p.C = C; p.z = (c.flags & MAMBA_SPEC_FLAG_GATE) ? io->z : nullptr; p.y = io->y;
     p.A = A; p.D = D; p.conv_w = io->conv_w; p.conv_b = io->conv_b;
+    p.row_off = nullptr; p.row_off_const = 0; p.row_off_cap = 0; p.n_prev_done = 0; p.n_prev_full = 0;
     p.dt_bias = (c.flags & MAMBA_SPEC_FLAG_DT_SOFTPLUS) ? io->dt_bias : nullptr;
     p.sel = (c.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS) ? ctx->d_sel : nullptr;
     p.state_k = (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? (float *)io->state_k : nullptr;
@@ -262,7 +268,109 @@ static int check_and_fill(mamba_spec_ctx *ctx, VerifyParams &p, void *state, voi
     return MAMBA_SPEC_OK;
 }
 
+static int launch_one(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who);
+
+// A token block of more than 16 rows, for the streaming kernel: segments of at most 16 rows, one launch each.
+// The first takes the pending tokens and as many drafts as fit, puts the state at the verified position back
+// into the cache (Sec. 4.3 iii) and leaves the state after its last token in a scratch buffer, from which the
+// next segment goes on with nothing pending, and so on; only the last writes a second snapshot if the caller
+// wants one.  (The same unrolled form, applied segment by segment; the per-token states still never exist.)
+static int launch_split(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
+    const mamba_spec_config &c = ctx->cfg;
+    const size_t n_state = (size_t)c.batch_max * c.n_heads * c.head_dim * c.d_state * sizeof(float);
+    const size_t n_conv = (size_t)c.batch_max * (c.conv_width - 1) * c.n_heads * c.head_dim * act_bytes(c);
+    if (!ctx->d_zero) {   // all or nothing
+        cudaError_t e = cudaSuccess;
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaMalloc(&ctx->split_state[i], n_state);
+            if (e == cudaSuccess) e = cudaMalloc(&ctx->split_conv[i], n_conv + 16);
+        }
+        int32_t *zero = nullptr;
+        if (e == cudaSuccess) e = cudaMalloc(&zero, sizeof(int32_t) * (size_t)c.batch_max);
+        if (e == cudaSuccess) e = cudaMemset(zero, 0, sizeof(int32_t) * (size_t)c.batch_max);
+        if (e != cudaSuccess) {
+            for (int i = 0; i < 2; ++i) {
+                if (ctx->split_state[i]) cudaFree(ctx->split_state[i]);
+                if (ctx->split_conv[i]) cudaFree(ctx->split_conv[i]);
+                ctx->split_state[i] = nullptr;
+                ctx->split_conv[i] = nullptr;
+            }
+            if (zero) cudaFree(zero);
+            return fail(ctx, MAMBA_SPEC_ERR_CUDA, "%s: scratch for a split token block: %s", who, cudaGetErrorString(e));
+        }
+        ctx->d_zero = zero;
+    }
+    const int kSeg = 16;
+    int done = 0, seg = 0;
+    const int k_first = kSeg - p.j_cap < p.k ? kSeg - p.j_cap : p.k;
+    while (done < p.k || seg == 0) {
+        const int k_i = seg == 0 ? k_first : (p.k - done < kSeg ? p.k - done : kSeg);
+        const bool last = done + k_i >= p.k;
+        VerifyParams q = p;
+        q.k = k_i;
+        if (seg > 0) {
+            q.state = ctx->split_state[(seg - 1) & 1];
+            q.conv_state = ctx->split_conv[(seg - 1) & 1];
+            q.n_prev = ctx->d_zero;
+            q.j_cap = 0;
+            q.n_prev_done = 0;
+            q.n_prev_full = 0;
+            q.row_off = p.n_prev;
+            q.row_off_cap = p.row_off_cap + p.j_cap;   // all of this sequence's pending rows come first
+            q.row_off_const = done;
+        }
+        if (!last) {
+            q.state_k = ctx->split_state[seg & 1];
+            q.conv_state_k = ctx->split_conv[seg & 1];
+        }
+        const int rc = launch_one(ctx, q, stream, who);
+        if (rc) return rc;
+        done += k_i;
+        ++seg;
+    }
+    return MAMBA_SPEC_OK;
+}
+
 static int launch(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
+    const mamba_spec_config &c = ctx->cfg;
+    const int kSeg = 16, kPend = 8;   // rows and pending rows that one launch of the streaming kernel takes
+    // more than 16 token rows: in segments, where the streaming kernel would take a segment of this shape
+    if (p.j_cap + p.k > kSeg && c.kernel_select != MAMBA_SPEC_KERNEL_GENERIC && p.sel == nullptr &&
+        !(p.flags & (kFlagYNewOnly | kFlagMamba1)) && ctx->map_cache.size() > 0) {
+        const bool bf16 = c.act_dtype == MAMBA_SPEC_DTYPE_BF16;
+        const int n_flush = p.j_cap > kPend ? (p.j_cap - 1) / kPend : 0;
+        VerifyParams rest = p;
+        if (n_flush > 0) {
+            rest.n_prev_full = p.j_cap;
+            rest.n_prev_done = kPend * n_flush;
+            rest.j_cap = p.j_cap - kPend * n_flush;
+            rest.row_off = p.n_prev;
+            rest.row_off_cap = kPend * n_flush;
+        }
+        VerifyParams probe = rest;
+        probe.k = rest.j_cap + p.k > kSeg ? kSeg - rest.j_cap : p.k;
+        VerifyParams probe_flush = p;
+        probe_flush.j_cap = kPend; probe_flush.k = 0; probe_flush.state_k = nullptr; probe_flush.conv_state_k = nullptr;
+        if (plan_verify_stream(probe, bf16, ctx->sm_count, ctx->smem_optin).ok &&
+            (n_flush == 0 || plan_verify_stream(probe_flush, bf16, ctx->sm_count, ctx->smem_optin).ok)) {
+            // more than 8 pending rows: the first ones are replayed 8 at a time, each launch advancing the cache
+            // in place (a call with no drafts), until at most 8 are left for the launch that takes the drafts
+            for (int i = 0; i < n_flush; ++i) {
+                VerifyParams q = probe_flush;
+                q.n_prev_full = p.j_cap;
+                q.n_prev_done = kPend * i;
+                q.row_off = p.n_prev;
+                q.row_off_cap = kPend * i;
+                const int rc = launch_one(ctx, q, stream, who);
+                if (rc) return rc;
+            }
+            return rest.j_cap + rest.k > kSeg ? launch_split(ctx, rest, stream, who) : launch_one(ctx, rest, stream, who);
+        }
+    }
+    return launch_one(ctx, p, stream, who);
+}
+
+static int launch_one(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
     const mamba_spec_config &c = ctx->cfg;
     const bool bf16 = c.act_dtype == MAMBA_SPEC_DTYPE_BF16;
     cudaError_t e;
@@ -661,6 +769,11 @@ void mamba_spec_destroy(mamba_spec_ctx *ctx) {
                 if (ctx->ring[i]) cudaFree(ctx->ring[i]);
                 if (ctx->slab[i]) cudaFree(ctx->slab[i]);
             }
+            for (int i = 0; i < 2; ++i) {
+                if (ctx->split_state[i]) cudaFree(ctx->split_state[i]);
+                if (ctx->split_conv[i]) cudaFree(ctx->split_conv[i]);
+            }
+            if (ctx->d_zero) cudaFree(ctx->d_zero);
             void *bufs[] = {ctx->d_n_prev, ctx->d_status, ctx->d_sel, ctx->st_x, ctx->st_dt, ctx->st_B, ctx->st_C,
                             ctx->st_z, ctx->st_y, ctx->st_n_prev};
             for (void *b : bufs)

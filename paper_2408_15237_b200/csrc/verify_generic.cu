@@ -45,6 +45,7 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
     act_t *cst = (act_t *)(swapped ? p.conv_state_k : p.conv_state), *cst_other = (act_t *)(swapped ? p.conv_state : p.conv_state_k);
     float *st_cur = swapped ? p.state_k : p.state, *st_other = swapped ? p.state : p.state_k;
     const int gB = h / (H / p.GB), gC = h / (H / p.GC);
+    const int row_first = first_row(p, b);
 
     float win[kMaxConvWidth - 1], tap[kMaxConvWidth];
 #pragma unroll
@@ -68,7 +69,7 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
     for (int i = 0; i < kRegs; ++i) hreg[i] = (lane + 32 * i < N) ? srow[lane + 32 * i] : 0.f;
 
     for (int t = 0; t < T; ++t) {
-        const size_t bt = (size_t)b * p.t_max + t;
+        const size_t bt = (size_t)b * p.t_max + row_first + t;
         const float xin = ld_act(x, (bt * H + h) * P + pr);
         float acc = bias;
 #pragma unroll

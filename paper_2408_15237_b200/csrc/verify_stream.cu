@@ -251,7 +251,7 @@ __device__ __forceinline__ bool issue_raw(const VerifyParams &p, const StreamLay
                                           uint32_t smem_base, Ctrl &ctl, int rs, int rp, int b, int h, int rc, int lane) {
     if (!mbar_wait(smem_u32(&ctl.raw_empty[rs]), (uint32_t)rp ^ 1u, &ctl.abort)) return false;
     const uint32_t raw = smem_base + L.raw_off + rs * L.raw_stride, bar = smem_u32(&ctl.raw_full[rs]);
-    const int c0 = h * p.P + rc * CR, row0 = b * p.t_max;
+    const int c0 = h * p.P + rc * CR, row0 = b * p.t_max + first_row(p, b);
 #ifdef MSPEC_TEST_RAW_NEVER_FULL
     // Test build only: one transaction byte more is expected than is requested, so every copy lands and the
     // barrier still never completes -- the consumers' bounded wait runs out.
@@ -673,7 +673,7 @@ __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const Stream
         const float *Gm = reinterpret_cast<const float *>(gb + L.c_G);
         // (with new rows only, y is [batch][k]: token j is its row 0 and the replayed rows' outputs are dropped)
         const bool y_new = (p.flags & kFlagYNewOnly) != 0;
-        const size_t y0 = (((size_t)b * (y_new ? p.k : p.t_max) - (y_new ? j : 0)) * p.H + h) * p.P + rc * CR;
+        const size_t y0 = (((size_t)b * (y_new ? p.k : p.t_max) - (y_new ? j : 0) + (y_new ? 0 : first_row(p, b))) * p.H + h) * p.P + rc * CR;
         const size_t tstride = (size_t)p.H * p.P;
         // a thread's elements share their row (the group's thread count is a multiple of CR): its xc values
         // are read once; D sits on the diagonal of G

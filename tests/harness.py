@@ -13,6 +13,7 @@ import oracle
 from paper_2408_15237_b200 import synth
 
 TOL = {"bf16": 2e-3, "fp32": 1e-5}   # max relative L2 error on y and on the committed state
+NAMED_WORKLOADS = {c.name for c in synth.CONFIGS.values()} | {c.name for c in synth.SWEEP.values()}
 
 
 def act_dtype(s):
@@ -93,6 +94,13 @@ class Layer:
             e_q = rel_l2(yg[valid], y_ref_q[valid])
             assert e_q <= tol, f"{what}: y rel L2 against the bf16-rounded oracle {e_q:.3e} > {tol}"
             assert e_y <= floor + 0.1 * tol, f"{what}: y rel L2 {e_y:.3e} vs rounding floor {floor:.3e}"
+            # and the stated tolerance taken literally, against the unrounded oracle, on the named workloads (the
+            # five configurations and the sweep).  Rounding the exact output to bf16 costs 1.4e-3 .. 1.7e-3 there;
+            # on the synthetic edge shapes it alone reaches 2.0e-3 .. 2.4e-3 (small state widths, few values), which
+            # the two checks above and the fp32-output tests cover instead.
+            if self.s.name in NAMED_WORKLOADS:
+                assert e_y <= tol, f"{what}: y rel L2 against the unrounded oracle {e_y:.3e} > {tol}"
+            self.last_unrounded = e_y
             e_y = e_q
         else:
             assert e_y <= tol, f"{what}: y rel L2 {e_y:.3e} > {tol}"
@@ -127,12 +135,14 @@ def run_rounds(s, rounds, kernel=0, layer=0, first_j=None, accept=None, final_fl
     stream = synth.token_stream(s, layer, rounds * s.k + s.k + fj + 1)
     r = synth.Rounds(s, stream, first_j=fj)
     worst = (0.0, 0.0)
+    run_rounds.worst_unrounded = 0.0   # largest rel L2 of a bf16 y against the UNROUNDED oracle (the figure the tolerance names)
     for rd in range(rounds):
         b = r.batch()
         y_gpu = lay.gpu_verify(ver, b, s.k)
         y_ref = lay.oracle_verify(b, s.k)
         e = lay.check(y_gpu, y_ref, tol, f"{s.name} round {rd} [{ver.last_kernel}]")
         worst = (max(worst[0], e[0]), max(worst[1], e[1]))
+        run_rounds.worst_unrounded = max(run_rounds.worst_unrounded, getattr(lay, "last_unrounded", e[0]))
         a = synth.acceptance(s, rd) if accept is None else np.asarray(accept(rd), dtype=np.int32)
         r.accept(a)
     if final_flush:

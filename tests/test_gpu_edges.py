@@ -227,7 +227,8 @@ def test_argument_errors_are_codes_not_crashes():
     v2.close()
 
 
-@pytest.mark.parametrize("step,kernel", [(1, STREAM), (2, STREAM), (16, STREAM), (16, GENERIC), (32, GENERIC)])
+@pytest.mark.parametrize("step,kernel", [(1, STREAM), (2, STREAM), (16, STREAM), (16, GENERIC), (32, GENERIC), (32, STREAM),
+                                         (24, STREAM)])
 def test_multistep_decoding_from_the_cached_state(step, kernel):
     """The paper's second use of the kernel (Fig. 3): no pending tokens, `step` new tokens per call, t_max = step.
     Three calls in a row; the cache must stay bit-for-bit untouched (nothing was accepted)."""
@@ -271,10 +272,14 @@ def test_draft_side_step_replays_the_accepted_tokens_and_decodes_one(kernel):
 
 
 LONG = synth.Shape("edge_long", Bt=3, H=8, P=64, N=128, GB=2, GC=8, W=4, k=8, act="bf16")
+# 20 new rows on top of up to 8 pending ones: a token block that the streaming kernel takes in segments
+BLOCK28 = synth.Shape("edge_block28", Bt=3, H=8, P=64, N=128, GB=2, GC=8, W=4, k=20, act="bf16", t_rows=28, k_prev=8)
+# and up to 20 pending ones (40 rows): the pending rows beyond 8 are replayed by launches of their own
+BLOCK40 = synth.Shape("edge_block40", Bt=5, H=8, P=64, N=128, GB=2, GC=8, W=4, k=20, act="bf16")
 
 
 @pytest.mark.parametrize("kernel", [GENERIC, STREAM])
-@pytest.mark.parametrize("s", [SMALL, SMALL64, LONG], ids=["n128", "n64", "k8"])
+@pytest.mark.parametrize("s", [SMALL, SMALL64, LONG, BLOCK28], ids=["n128", "n64", "k8", "k20"])
 def test_second_snapshot_after_all_tokens(s, kernel):
     """MAMBA_SPEC_FLAG_STATE_K (Algorithm 2 caches h_j and h_k): besides the cache at the verified position j
     the call leaves the cache after all T_b = j_b + k tokens in a second pair of buffers.  The oracle for the
@@ -286,7 +291,8 @@ def test_second_snapshot_after_all_tokens(s, kernel):
     lay = h.Layer(s)
     ad = h.act_dtype(s)
     r = synth.Rounds(s, synth.token_stream(s, 0, 48))
-    pend = [np.arange(s.Bt) % (s.k + 1), np.zeros(s.Bt), np.full(s.Bt, s.k)]
+    cap = s.k_prev if s.k_prev else s.k
+    pend = [np.arange(s.Bt) % (cap + 1), np.zeros(s.Bt), np.full(s.Bt, cap)]
     for call, n_prev in enumerate(pend):
         n_prev = n_prev.astype(np.int32)
         r.cursor, r.n_prev = (r.cursor + n_prev if call else n_prev.astype(np.int64)), n_prev.copy()
@@ -362,3 +368,16 @@ def test_checkpoint_and_resume_in_a_fresh_context(kernel):
     assert torch.equal(lay_b.state, want_state) and torch.equal(lay_b.conv, want_conv)
     assert ver_b.status() == 0
     ver_b.close()
+
+
+@pytest.mark.parametrize("kernel", [GENERIC, STREAM])
+@pytest.mark.parametrize("s", [BLOCK28, BLOCK40], ids=["pending8", "pending20"])
+def test_token_blocks_longer_than_sixteen_rows_with_pending_tokens(s, kernel):
+    """20 new tokens per call on top of up to 8 (28 rows) or up to 20 (40 rows) pending ones: the streaming
+    kernel takes such a block in launches of at most 16 rows with at most 8 pending ones, carrying the state from
+    one to the next; outputs in float32 so that the bound is the arithmetic's 1e-5.  Four rounds with mixed
+    acceptance, then a call with no drafts that only replays the pending rows."""
+    h = H()
+    worst, name = h.run_rounds(s, 4, kernel=kernel, first_j=5, y_f32=True, tol=1e-5, final_flush=True)
+    assert ("stream" in name) == (kernel == STREAM)
+    assert max(worst) <= 1e-5
