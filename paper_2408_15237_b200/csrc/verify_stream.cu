@@ -246,12 +246,12 @@ __device__ __forceinline__ int pending_of(const VerifyParams &p, const Ctrl &ctl
 // Requests the small inputs of one chunk: nine TMA requests issued by nine lanes (x, z, B, C, dt and
 // the conv window through tensor maps, each covering all TCAP token rows; taps and bias as plain bulk
 // copies).  Rows beyond the sequence's T tokens are fetched but never used.
-template <int N, int CR>
+template <int N, int CR, bool EXT>
 __device__ __forceinline__ bool issue_raw(const VerifyParams &p, const StreamLayout &L, const InputMaps &tm,
                                           uint32_t smem_base, Ctrl &ctl, int rs, int rp, int b, int h, int rc, int lane) {
     if (!mbar_wait(smem_u32(&ctl.raw_empty[rs]), (uint32_t)rp ^ 1u, &ctl.abort)) return false;
     const uint32_t raw = smem_base + L.raw_off + rs * L.raw_stride, bar = smem_u32(&ctl.raw_full[rs]);
-    const int c0 = h * p.P + rc * CR, row0 = b * p.t_max + first_row(p, b);
+    const int c0 = h * p.P + rc * CR, row0 = b * p.t_max + (EXT ? first_row(p, b) : 0);
 #ifdef MSPEC_TEST_RAW_NEVER_FULL
     // Test build only: one transaction byte more is expected than is requested, so every copy lands and the
     // barrier still never completes -- the consumers' bounded wait runs out.
@@ -270,7 +270,7 @@ __device__ __forceinline__ bool issue_raw(const VerifyParams &p, const StreamLay
         const uint32_t dst = raw + (lane == 0 ? L.r_x : lane == 1 ? L.r_z : lane == 2 ? L.r_B : lane == 3 ? L.r_C
                                                                    : lane == 4 ? L.r_dt : L.r_cst);
         // (commit-selects mode: the conv window comes from whichever buffer holds this sequence's cache)
-        const TensorMapBytes *map = (lane == 5 && p.sel != nullptr && p.sel[b] != 0) ? &tm.cst_k : &tm.x + lane;
+        const TensorMapBytes *map = (EXT && lane == 5 && p.sel != nullptr && p.sel[b] != 0) ? &tm.cst_k : &tm.x + lane;
         if (lane != 1 || p.z != nullptr) tma_load_2d(dst, as_map(map), cx, cy, bar);
     } else if (lane < 8) {
         const bool taps = lane == 6;
@@ -282,7 +282,7 @@ __device__ __forceinline__ bool issue_raw(const VerifyParams &p, const StreamLay
 
 // The small inputs of a chunk are requested `lead` chunks before its state rows: they feed the
 // prologue, whose results are needed at the moment the state lands.
-template <int N, int CR>
+template <int N, int CR, bool EXT>
 __device__ __forceinline__ void producer_role(const VerifyParams &p, const StreamLayout &L, unsigned char *smem,
                                               Ctrl &ctl, const InputMaps &tm, int lane) {
     constexpr uint32_t kStateBytes = CR * N * 4;
@@ -294,7 +294,7 @@ __device__ __forceinline__ void producer_role(const VerifyParams &p, const Strea
     for (int it = 0; it < nmine; ++it) {
         const int rlim = it + L.lead + 1 < nmine ? it + L.lead + 1 : nmine;
         for (; itr < rlim; ++itr) {
-            if (!issue_raw<N, CR>(p, L, tm, smem_base, ctl, rs, rp, pr.b, pr.h, pr.rc, lane)) {
+            if (!issue_raw<N, CR, EXT>(p, L, tm, smem_base, ctl, rs, rp, pr.b, pr.h, pr.rc, lane)) {
                 atomicOr(p.status, kStatusCopyTimeout);
                 ctl.abort = 1;
                 return;
@@ -312,7 +312,7 @@ __device__ __forceinline__ void producer_role(const VerifyParams &p, const Strea
                 const uint32_t sbar = smem_u32(&ctl.state_full[ss]);
                 ctl.state_par[ss] = sp;
                 mbar_arrive_expect_tx(sbar, kStateBytes);
-                const bool swapped = p.sel != nullptr && p.sel[ps.b] != 0;   // commit-selects mode: where this sequence's cache is
+                const bool swapped = EXT && p.sel != nullptr && p.sel[ps.b] != 0;   // commit-selects mode: where this sequence's cache is
                 tma_load_3d(smem_base + L.state_off + ss * L.state_stride, as_map(swapped ? &tm.state_k : &tm.state), 0, ps.q * CR, 0, sbar);
             }
         }
@@ -334,7 +334,7 @@ __device__ __forceinline__ void producer_role(const VerifyParams &p, const Strea
 //   gate    SiLU(z_t), same mapping; conv window at position j -> global (Sec. 4.3 iii)
 //   rows    fp32 copies of the C rows and of the B rows s < j, which the stream phase reads as broadcasts
 //   decay   alpha_t, wsp_s, alpha_j by the lanes of the warp before the last
-template <int N, int CR, bool SNAP>
+template <int N, int CR, bool SNAP, bool EXT>
 __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const StreamLayout &L, const unsigned char *raw,
                                                unsigned char *gb, int b, int h, int rc, int j, int T,
                                                float A_of_head, float D_of_head, int gtid, bool swapped) {
@@ -348,7 +348,7 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
     float *xcs = reinterpret_cast<float *>(gb + L.c_xc);  // [t][CR]
     const unsigned short *dtr = reinterpret_cast<const unsigned short *>(raw + L.r_dt) + (h & 7);   // dt_t at [t * 8]
     // the sampling interval of token r: as it arrives, or softplus(raw + bias) when it arrives raw (Sec. 2.2)
-    const bool dt_raw = (p.flags & kFlagDtSoftplus) != 0;
+    const bool dt_raw = EXT && (p.flags & kFlagDtSoftplus) != 0;
     const float dt_b = (dt_raw && p.dt_bias != nullptr) ? p.dt_bias[h] : 0.f;
     auto dt_at = [&](int r) {
         const float v = bf16_bits_to_f32(dtr[r * 8]);
@@ -518,7 +518,7 @@ __device__ __forceinline__ void prologue_phase(const VerifyParams &p, const Stre
 // broadcasts) goes to shared memory; after a group barrier the quarters are summed and y is formed
 // with fully coalesced stores.  Where tokens were accepted the state at position j is formed in the
 // same registers, written back into the stage and stored to global memory by one TMA request.
-template <int N, int CR, bool SNAP>
+template <int N, int CR, bool SNAP, bool EXT>
 __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const StreamLayout &L, const InputMaps &tm,
                                              unsigned char *st, unsigned char *gb, uint32_t empty_bar, int bar_id, int q,
                                              int b, int h, int rc, int j, int T, int gtid, bool swapped) {
@@ -672,8 +672,8 @@ __device__ __forceinline__ bool stream_phase(const VerifyParams &p, const Stream
         const float *xcs = reinterpret_cast<const float *>(gb + L.c_xc), *gz = reinterpret_cast<const float *>(gb + L.c_gz);
         const float *Gm = reinterpret_cast<const float *>(gb + L.c_G);
         // (with new rows only, y is [batch][k]: token j is its row 0 and the replayed rows' outputs are dropped)
-        const bool y_new = (p.flags & kFlagYNewOnly) != 0;
-        const size_t y0 = (((size_t)b * (y_new ? p.k : p.t_max) - (y_new ? j : 0) + (y_new ? 0 : first_row(p, b))) * p.H + h) * p.P + rc * CR;
+        const bool y_new = EXT && (p.flags & kFlagYNewOnly) != 0;
+        const size_t y0 = (((size_t)b * (y_new ? p.k : p.t_max) - (y_new ? j : 0) + ((y_new || !EXT) ? 0 : first_row(p, b))) * p.H + h) * p.P + rc * CR;
         const size_t tstride = (size_t)p.H * p.P;
         // a thread's elements share their row (the group's thread count is a multiple of CR): its xc values
         // are read once; D sits on the diagonal of G
@@ -731,7 +731,7 @@ __device__ __forceinline__ bool named_bar_and(int id, int n, bool pred) {
     return r != 0;
 }
 
-template <int N, int CR, bool SNAP>
+template <int N, int CR, bool SNAP, bool EXT>
 __device__ __forceinline__ void compute_role(const VerifyParams &p, const StreamLayout &L, unsigned char *smem, Ctrl &ctl,
                                              const InputMaps &tm, int group, int gtid) {
     const int lane = gtid & 31, bar_id = 1 + group;
@@ -747,21 +747,21 @@ __device__ __forceinline__ void compute_role(const VerifyParams &p, const Stream
     ring_advance(rs, rp, group, L.R);
     for (; it < nmine; it += L.ngroups) {
         const int j = pending_of(p, ctl, x.b), T = j + p.k;
-        const bool swapped = SNAP && p.sel != nullptr && p.sel[x.b] != 0;   // commit-selects mode: the cache is in the second buffers
+        const bool swapped = EXT && SNAP && p.sel != nullptr && p.sel[x.b] != 0;   // commit-selects mode: the cache is in the second buffers
         // the group's buffer is free once every warp has left the previous chunk; the inputs must be in
         bool ok = mbar_wait(smem_u32(&ctl.raw_full[rs]), (uint32_t)rp, &ctl.abort);
         ok = named_bar_and(bar_id, kGroupThreads, ok);
         if (!ok) break;
         if (store_pending) { release_stage(pending_bar); store_pending = false; }
         const unsigned char *raw = smem + L.raw_off + (size_t)rs * L.raw_stride;
-        prologue_phase<N, CR, SNAP>(p, L, raw, gb, x.b, x.h, x.rc, j, T, ctl.A[x.h], ctl.D[x.h], gtid, swapped);
+        prologue_phase<N, CR, SNAP, EXT>(p, L, raw, gb, x.b, x.h, x.rc, j, T, ctl.A[x.h], ctl.D[x.h], gtid, swapped);
         ok = mbar_wait(smem_u32(&ctl.state_full[ss]), (uint32_t)sp, &ctl.abort);
         ok = named_bar_and(bar_id, kGroupThreads, ok);   // also: the group's buffer is complete
         if (lane == 0) mbar_arrive(smem_u32(&ctl.raw_empty[rs]));
         if (!ok) break;
         unsigned char *st = smem + L.state_off + (size_t)ss * L.state_stride;
         pending_bar = smem_u32(&ctl.state_empty[ss]);
-        store_pending = stream_phase<N, CR, SNAP>(p, L, tm, st, gb, pending_bar, bar_id, x.q, x.b, x.h, x.rc, j, T, gtid, swapped);
+        store_pending = stream_phase<N, CR, SNAP, EXT>(p, L, tm, st, gb, pending_bar, bar_id, x.q, x.b, x.h, x.rc, j, T, gtid, swapped);
         advance(x, wi.grp, H, cph);
         ring_advance(ss, sp, L.ngroups, L.S);
         ring_advance(rs, rp, L.ngroups, L.R);
@@ -774,7 +774,7 @@ __device__ __forceinline__ void compute_role(const VerifyParams &p, const Stream
 }
 
 // ---------------------------------------------------------------- the kernel
-template <int N, int CR, bool SNAP>
+template <int N, int CR, bool SNAP, bool EXT>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_constant__ StreamLayout L,
                      const __grid_constant__ InputMaps tm) {
@@ -842,7 +842,7 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
     // with this kernel but with nothing older.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (is_producer) {
-        producer_role<N, CR>(p, L, smem, ctl, tm, lane);
+        producer_role<N, CR, EXT>(p, L, smem, ctl, tm, lane);
     } else {
         constexpr int kComputeThreads = kGroups * kGroupThreads;
         const int ntab = p.batch < kJTable ? p.batch : kJTable;
@@ -851,7 +851,7 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
 #pragma unroll 1
         for (int i = tid; i < p.H; i += kComputeThreads) { ctl.A[i] = p.A[i]; ctl.D[i] = p.D[i]; }
         named_bar_sync(15, kComputeThreads);
-        compute_role<N, CR, SNAP>(p, L, smem, ctl, tm, warp / kGroupWarps, tid % kGroupThreads);
+        compute_role<N, CR, SNAP, EXT>(p, L, smem, ctl, tm, warp / kGroupWarps, tid % kGroupThreads);
     }
 
     __syncthreads();
@@ -911,9 +911,9 @@ bool encode_state(EncodeTiledFn fn, TensorMapBytes *map, const void *base, size_
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int N, int CR, bool SNAP>
+template <int N, int CR, bool SNAP, bool EXT>
 cudaError_t launch_variant(const VerifyParams &p, const StreamPlan &plan, const InputMaps &tm, cudaStream_t stream) {
-    auto kern = verify_stream_kernel<N, CR, SNAP>;
+    auto kern = verify_stream_kernel<N, CR, SNAP, EXT>;
     static size_t configured[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -1035,10 +1035,12 @@ StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, si
 
     plan.ok = true;
     plan.grid = (int)grid;
-    plan.variant = (N == 128 ? 0 : 2) + (CR == 64 ? 0 : 1) + (p.state_k != nullptr ? 4 : 0);
+    const bool ext = (p.flags & (kFlagDtSoftplus | kFlagYNewOnly)) != 0 || p.sel != nullptr || p.row_off != nullptr ||
+                     p.row_off_const != 0;
+    plan.variant = (N == 128 ? 0 : 2) + (CR == 64 ? 0 : 1) + (p.state_k != nullptr ? 4 : 0) + (ext ? 8 : 0);
     plan.smem_bytes = (size_t)L.grp_off + (size_t)L.ngroups * L.grp_stride;
-    snprintf(plan.name, sizeof plan.name, "stream<N=%d,CR=%d,groups=%d,TCAP=%d,S=%d,R=%d,lead=%d,grid=%d>", N, CR, L.ngroups,
-             L.TCAP, L.S, L.R, L.lead, (int)grid);
+    snprintf(plan.name, sizeof plan.name, "stream<N=%d,CR=%d,groups=%d,TCAP=%d,S=%d,R=%d,lead=%d,grid=%d%s>", N, CR, L.ngroups,
+             L.TCAP, L.S, L.R, L.lead, (int)grid, ext ? ",ext" : "");
     return plan;
 }
 
@@ -1065,16 +1067,20 @@ bool encode_stream_maps(const VerifyParams &p, const StreamPlan &plan, InputMaps
 }
 
 cudaError_t launch_verify_stream(const VerifyParams &p, const StreamPlan &plan, const InputMaps &tm, cudaStream_t stream) {
-    switch (plan.variant) {   // bit 0: 32-row chunks; bit 1: N = 64; bit 2: second snapshot
-        case 0: return launch_variant<128, 64, false>(p, plan, tm, stream);
-        case 1: return launch_variant<128, 32, false>(p, plan, tm, stream);
-        case 2: return launch_variant<64, 64, false>(p, plan, tm, stream);
-        case 3: return launch_variant<64, 32, false>(p, plan, tm, stream);
-        case 4: return launch_variant<128, 64, true>(p, plan, tm, stream);
-        case 5: return launch_variant<128, 32, true>(p, plan, tm, stream);
-        case 6: return launch_variant<64, 64, true>(p, plan, tm, stream);
-        case 7: return launch_variant<64, 32, true>(p, plan, tm, stream);
+    // bit 0: 32-row chunks; bit 1: N = 64; bit 2: second snapshot; bit 3: the variants of the call (raw interval,
+    // cache in either of two buffers, outputs for new rows only, rows at an offset) compiled in
+    switch (plan.variant) {
+#define MSPEC_CASE(v, n, cr, snap, ext) case v: return launch_variant<n, cr, snap, ext>(p, plan, tm, stream);
+        MSPEC_CASE(0, 128, 64, false, false) MSPEC_CASE(1, 128, 32, false, false)
+        MSPEC_CASE(2, 64, 64, false, false) MSPEC_CASE(3, 64, 32, false, false)
+        MSPEC_CASE(4, 128, 64, true, false) MSPEC_CASE(5, 128, 32, true, false)
+        MSPEC_CASE(6, 64, 64, true, false) MSPEC_CASE(7, 64, 32, true, false)
+        MSPEC_CASE(8, 128, 64, false, true) MSPEC_CASE(9, 128, 32, false, true)
+        MSPEC_CASE(10, 64, 64, false, true) MSPEC_CASE(11, 64, 32, false, true)
+        MSPEC_CASE(12, 128, 64, true, true) MSPEC_CASE(13, 128, 32, true, true)
+        MSPEC_CASE(14, 64, 64, true, true) MSPEC_CASE(15, 64, 32, true, true)
         default: return cudaErrorInvalidValue;
+#undef MSPEC_CASE
     }
 }
 
