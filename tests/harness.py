@@ -13,7 +13,6 @@ import oracle
 from paper_2408_15237_b200 import synth
 
 TOL = {"bf16": 2e-3, "fp32": 1e-5}   # max relative L2 error on y and on the committed state
-NAMED_WORKLOADS = {c.name for c in synth.CONFIGS.values()} | {c.name for c in synth.SWEEP.values()}
 
 
 def act_dtype(s):
@@ -94,11 +93,12 @@ class Layer:
             e_q = rel_l2(yg[valid], y_ref_q[valid])
             assert e_q <= tol, f"{what}: y rel L2 against the bf16-rounded oracle {e_q:.3e} > {tol}"
             assert e_y <= floor + 0.1 * tol, f"{what}: y rel L2 {e_y:.3e} vs rounding floor {floor:.3e}"
-            # and the stated tolerance taken literally, against the unrounded oracle, on the named workloads (the
-            # five configurations and the sweep).  Rounding the exact output to bf16 costs 1.4e-3 .. 1.7e-3 there;
-            # on the synthetic edge shapes it alone reaches 2.0e-3 .. 2.4e-3 (small state widths, few values), which
-            # the two checks above and the fp32-output tests cover instead.
-            if self.s.name in NAMED_WORKLOADS:
+            # and the stated tolerance taken literally, against the unrounded oracle, wherever rounding the exact output
+            # to bf16 leaves room for it.  That rounding alone costs 1.4e-3 .. 1.8e-3 on the large workloads and
+            # 2.0e-3 .. 2.4e-3 where few values are compared (batch 1 with two drafts, the small edge shapes): there
+            # a perfect kernel exceeds 2e-3, and the two checks above and the fp32-output tests stand in.
+            self.last_floor = floor
+            if floor <= 0.9 * tol:
                 assert e_y <= tol, f"{what}: y rel L2 against the unrounded oracle {e_y:.3e} > {tol}"
             self.last_unrounded = e_y
             e_y = e_q
