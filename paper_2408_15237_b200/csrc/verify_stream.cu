@@ -812,6 +812,8 @@ verify_stream_kernel(const __grid_constant__ VerifyParams p, const __grid_consta
     // first (no architectural effect: they take cold misses off the path).  First state requests ahead of the
     // wait, for callers that can promise an unrelated previous kernel, were measured and lost 5 %.
     if (is_producer) {
+        // the nine tensor maps into the descriptor cache, so that the first requests do not wait for them
+        if (lane < 9) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<const void *>(&tm.x + lane)) : "memory");
         const WalkInfo &wi = *reinterpret_cast<const WalkInfo *>(ctl.walk);
         const Pos x0 = wi.start[0];
         const size_t trow = ((size_t)x0.b * p.t_max + (lane < p.t_max ? lane : 0)) ;
