@@ -137,7 +137,11 @@ typedef struct {
  * allocates the context.  Does not touch any caller tensor. */
 int mamba_spec_init(const mamba_spec_config *cfg, mamba_spec_ctx **out);
 
-/* The verification call described at the top of this file.  One kernel launch.
+/* The verification call described at the top of this file.  One kernel launch -- except that the streaming
+ * kernel takes at most 16 token rows of a sequence, of which at most 8 pending, per launch: a longer block
+ * (j_b + k_draft up to t_max) runs as several launches that carry the state from one to the next (Sec. 4.2: the
+ * same recurrence, applied piecewise; scratch for the carried state is allocated on the first such call; not
+ * combined with FLAG_COMMIT_SELECTS or FLAG_MAMBA1, which run such blocks in the generic kernel).
  *   state           [batch][H][P][N] float32, in/out: h_i -> h_{i+j_b}
  *   conv_state      [batch][W-1][H*P] act dtype, in/out, oldest row first
  *   x               [batch][t_max][H][P] act dtype, pre-conv inputs
