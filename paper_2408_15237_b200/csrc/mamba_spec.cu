@@ -331,40 +331,65 @@ static int launch_split(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t
     return MAMBA_SPEC_OK;
 }
 
+// How a call is launched: as one kernel, or -- a token block of more than 16 rows, where the streaming kernel would
+// take its pieces -- as `pending_only` launches that replay 8 pending rows each and then the rest in pieces of at
+// most 16 rows (launch_split).
+struct SplitPlan {
+    bool split;
+    int pending_only;     // launches without drafts that advance the cache over 8 pending rows each
+    int launches;         // all launches of the call
+    VerifyParams rest;    // the call that is left after them
+    StreamPlan first;     // plan of the first launch that takes drafts
+};
+static const int kSegRows = 16, kSegPending = 8;   // rows and pending rows that one launch of the streaming kernel takes
+
+static SplitPlan plan_split(const VerifyParams &p, const mamba_spec_config &c, int sm_count, size_t smem_optin) {
+    SplitPlan sp;
+    sp.split = false; sp.pending_only = 0; sp.launches = 1; sp.rest = p;
+    if (p.j_cap + p.k <= kSegRows || c.kernel_select == MAMBA_SPEC_KERNEL_GENERIC || p.sel != nullptr ||
+        (p.flags & (kFlagYNewOnly | kFlagMamba1)))
+        return sp;
+    const bool bf16 = c.act_dtype == MAMBA_SPEC_DTYPE_BF16;
+    const int n_flush = p.j_cap > kSegPending ? (p.j_cap - 1) / kSegPending : 0;
+    VerifyParams rest = p;
+    if (n_flush > 0) {
+        rest.n_prev_full = p.j_cap;
+        rest.n_prev_done = kSegPending * n_flush;
+        rest.j_cap = p.j_cap - kSegPending * n_flush;
+        rest.row_off = p.n_prev;
+        rest.row_off_cap = kSegPending * n_flush;
+    }
+    VerifyParams probe = rest;
+    probe.k = rest.j_cap + p.k > kSegRows ? kSegRows - rest.j_cap : p.k;
+    VerifyParams probe_flush = p;
+    probe_flush.j_cap = kSegPending; probe_flush.k = 0; probe_flush.state_k = nullptr; probe_flush.conv_state_k = nullptr;
+    sp.first = plan_verify_stream(probe, bf16, sm_count, smem_optin);
+    if (!sp.first.ok || (n_flush > 0 && !plan_verify_stream(probe_flush, bf16, sm_count, smem_optin).ok)) return sp;
+    sp.split = true;
+    sp.pending_only = n_flush;
+    sp.rest = rest;
+    const int k_first = kSegRows - rest.j_cap < rest.k ? kSegRows - rest.j_cap : rest.k;
+    sp.launches = n_flush + 1 + (rest.k - k_first + kSegRows - 1) / kSegRows;
+    return sp;
+}
+
 static int launch(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
-    const mamba_spec_config &c = ctx->cfg;
-    const int kSeg = 16, kPend = 8;   // rows and pending rows that one launch of the streaming kernel takes
-    // more than 16 token rows: in segments, where the streaming kernel would take a segment of this shape
-    if (p.j_cap + p.k > kSeg && c.kernel_select != MAMBA_SPEC_KERNEL_GENERIC && p.sel == nullptr &&
-        !(p.flags & (kFlagYNewOnly | kFlagMamba1)) && ctx->map_cache.size() > 0) {
-        const bool bf16 = c.act_dtype == MAMBA_SPEC_DTYPE_BF16;
-        const int n_flush = p.j_cap > kPend ? (p.j_cap - 1) / kPend : 0;
-        VerifyParams rest = p;
-        if (n_flush > 0) {
-            rest.n_prev_full = p.j_cap;
-            rest.n_prev_done = kPend * n_flush;
-            rest.j_cap = p.j_cap - kPend * n_flush;
-            rest.row_off = p.n_prev;
-            rest.row_off_cap = kPend * n_flush;
-        }
-        VerifyParams probe = rest;
-        probe.k = rest.j_cap + p.k > kSeg ? kSeg - rest.j_cap : p.k;
-        VerifyParams probe_flush = p;
-        probe_flush.j_cap = kPend; probe_flush.k = 0; probe_flush.state_k = nullptr; probe_flush.conv_state_k = nullptr;
-        if (plan_verify_stream(probe, bf16, ctx->sm_count, ctx->smem_optin).ok &&
-            (n_flush == 0 || plan_verify_stream(probe_flush, bf16, ctx->sm_count, ctx->smem_optin).ok)) {
+    if (ctx->map_cache.size() > 0) {   // (a context that may allocate: the carried state needs scratch)
+        const SplitPlan sp = plan_split(p, ctx->cfg, ctx->sm_count, ctx->smem_optin);
+        if (sp.split) {
             // more than 8 pending rows: the first ones are replayed 8 at a time, each launch advancing the cache
             // in place (a call with no drafts), until at most 8 are left for the launch that takes the drafts
-            for (int i = 0; i < n_flush; ++i) {
-                VerifyParams q = probe_flush;
+            for (int i = 0; i < sp.pending_only; ++i) {
+                VerifyParams q = p;
+                q.j_cap = kSegPending; q.k = 0; q.state_k = nullptr; q.conv_state_k = nullptr;
                 q.n_prev_full = p.j_cap;
-                q.n_prev_done = kPend * i;
+                q.n_prev_done = kSegPending * i;
                 q.row_off = p.n_prev;
-                q.row_off_cap = kPend * i;
+                q.row_off_cap = kSegPending * i;
                 const int rc = launch_one(ctx, q, stream, who);
                 if (rc) return rc;
             }
-            return rest.j_cap + rest.k > kSeg ? launch_split(ctx, rest, stream, who) : launch_one(ctx, rest, stream, who);
+            return sp.rest.j_cap + sp.rest.k > kSegRows ? launch_split(ctx, sp.rest, stream, who) : launch_one(ctx, sp.rest, stream, who);
         }
     }
     return launch_one(ctx, p, stream, who);
@@ -744,8 +769,11 @@ int mamba_spec_describe_plan(const mamba_spec_config *cfg, int32_t batch, int32_
     p.state_k = (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? (float *)buf : nullptr;
     const bool bf16 = c.act_dtype == MAMBA_SPEC_DTYPE_BF16;
     if (c.kernel_select != MAMBA_SPEC_KERNEL_GENERIC) {
-        const StreamPlan plan = plan_verify_stream(p, bf16, sm_count, (size_t)smem_per_block);
-        if (plan.ok) snprintf(buf, (size_t)buf_len, "%s", plan.name);
+        if (c.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS) p.sel = reinterpret_cast<const int32_t *>(buf);
+        const SplitPlan sp = plan_split(p, c, sm_count, (size_t)smem_per_block);
+        const StreamPlan plan = sp.split ? sp.first : plan_verify_stream(p, bf16, sm_count, (size_t)smem_per_block);
+        if (sp.split) snprintf(buf, (size_t)buf_len, "split(launches=%d,pending_only=%d) first %s", sp.launches, sp.pending_only, plan.name);
+        else if (plan.ok) snprintf(buf, (size_t)buf_len, "%s", plan.name);
         else snprintf(buf, (size_t)buf_len, "generic (%s)", plan.name);
     } else {
         snprintf(buf, (size_t)buf_len, "generic (selected)");

@@ -33,7 +33,7 @@ def test_benchmark_shape_gets_the_streaming_kernel(binding):
 
 @pytest.mark.parametrize("over,why", [(dict(act_dtype=0), "bf16"), (dict(conv_width=3), "conv width"), (dict(d_state=96), "state dim"),
                                       (dict(head_dim=48), "head dim"), (dict(n_heads=4, n_groups_b=1, n_groups_c=1), "head count"),
-                                      (dict(k_max=12), "token rows"), (dict(flags=1 | 2 | 16), "Mamba-1")])
+                                      (dict(flags=1 | 2 | 16), "Mamba-1")])
 def test_shapes_outside_the_streaming_kernel_fall_to_the_generic_one(binding, over, why):
     c = cfg(binding, **over)
     plan = binding.mamba_spec_describe_plan(c, 16, 2 * c.k_max, c.k_max, **B200)
@@ -73,3 +73,21 @@ def test_ring_invariant_over_the_supported_shapes(binding):
 def test_a_small_shared_memory_budget_is_refused_not_overrun(binding):
     plan = binding.mamba_spec_describe_plan(cfg(binding), 16, 8, 4, sm_count=148, smem_per_block=48 * 1024)
     assert plan.startswith("generic (") and "shared memory" in plan
+
+
+@pytest.mark.parametrize("k_max,t_max,k,launches,pending_only", [(12, 24, 12, 2, 1), (20, 28, 20, 2, 0), (20, 40, 20, 4, 2),
+                                                                  (32, 32, 32, 2, 0), (20, 28, 0, 3, 2)])
+def test_long_token_blocks_are_split_into_streaming_launches(binding, k_max, t_max, k, launches, pending_only):
+    """More than 16 token rows (or more than 8 pending ones): launches that replay 8 pending rows each, then the rest in
+    pieces of at most 16 rows; the first of those is planned like any call of its shape."""
+    plan = binding.mamba_spec_describe_plan(cfg(binding, k_max=k_max), 16, t_max, k, **B200)
+    f = fields(plan)
+    assert plan.startswith("split(") and "stream<" in plan, plan
+    assert f["launches"] == launches and f["pending_only"] == pending_only
+    assert f["TCAP"] <= 16
+
+
+def test_long_token_blocks_stay_whole_where_the_streaming_kernel_would_not_take_the_pieces(binding):
+    for over in (dict(flags=1 | 2 | 16), dict(flags=1 | 2 | 8 | 64), dict(kernel_select=1), dict(act_dtype=0)):
+        plan = binding.mamba_spec_describe_plan(cfg(binding, k_max=20, **over), 16, 40, 20, **B200)
+        assert plan.startswith("generic ("), plan
