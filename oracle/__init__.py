@@ -181,6 +181,24 @@ def softplus_dt(dt_raw, bias):
     return np.where(v > 30.0, v, np.log1p(np.exp(np.minimum(v, 30.0))))
 
 
+def gated_rmsnorm(y, weight, eps):
+    """The output normalisation of the Mamba-2 blocks that the hybrid Mamba2 models (Sec. 5) are made of: with
+    ``y`` the gated output of the verification call, ``[..., H, P]``, every token row is scaled to unit mean
+    square over its ``H*P`` channels and multiplied by a learned per-channel weight,
+    ``out[c] = weight[c] * y[c] / sqrt(mean_c(y[c]^2) + eps)``.  Rows that hold NaN (padding) stay NaN.
+    The paper does not print this formula; it is the published Mamba-2 block's (parity unpinned by the paper)."""
+    y = np.asarray(y, dtype=np.float64)
+    w = np.asarray(weight, dtype=np.float64).reshape(-1)
+    rows = y.reshape(-1, y.shape[-2] * y.shape[-1])
+    if rows.shape[1] != w.shape[0]:
+        raise ValueError("gated_rmsnorm: weight must have H*P entries")
+    out = np.empty_like(rows)
+    for r in range(rows.shape[0]):          # one token at a time, as the definition reads
+        mean_square = np.sum(rows[r] * rows[r]) / rows.shape[1]
+        out[r] = w * rows[r] / np.sqrt(mean_square + float(eps))
+    return out.reshape(y.shape)
+
+
 def verify_m1(state, conv_state, x, dt, Bm, Cm, A, D, conv_w, conv_b, z, n_prev, k, flags, threads=1):
     """Multi-step verification in the Mamba-1 parameterisation (Algorithm 1; Sec. 2.2): ``dt`` is
     ``[Bt, Tmax, H*P]``, ``A`` is ``[H*P, N]``, ``D`` is ``[H*P]``.  Returns ``(y, state_out, conv_state_out)``."""

@@ -442,3 +442,42 @@ def test_softplus_dt_against_its_identities():
     np.testing.assert_allclose((oracle.softplus_dt(v + eps, bias) - oracle.softplus_dt(v - eps, bias)) / (2 * eps),
                                1.0 / (1.0 + np.exp(-u)), rtol=1e-6, atol=1e-9)
     assert oracle.softplus_dt(np.array([100.0]), np.array([0.0]))[0] == 100.0
+
+
+# --------------------------------------------------------------------------- gated RMSNorm epilogue
+def test_gated_rmsnorm_against_its_definition_and_invariants():
+    rng = np.random.default_rng(7)
+    H, P = 3, 5
+    y = rng.standard_normal((2, 4, H, P))
+    w = 1.0 + 0.1 * rng.standard_normal(H * P)
+    eps = 1e-5
+    out = oracle.gated_rmsnorm(y, w, eps)
+    # the definition, element by element in plain Python
+    for b in range(2):
+        for t in range(4):
+            flat = [float(y[b, t, h, p]) for h in range(H) for p in range(P)]
+            ms = sum(v * v for v in flat) / len(flat)
+            for c, v in enumerate(flat):
+                assert abs(out[b, t, c // P, c % P] - w[c] * v / (ms + eps) ** 0.5) < 1e-13
+    # unit weight, no eps: every row has mean square exactly one
+    unit = oracle.gated_rmsnorm(y, np.ones(H * P), 0.0)
+    np.testing.assert_allclose((unit.reshape(8, -1) ** 2).mean(axis=1), 1.0, rtol=1e-13)
+    # scale invariance without eps, and the sign of the input survives
+    np.testing.assert_allclose(oracle.gated_rmsnorm(37.0 * y, w, 0.0), oracle.gated_rmsnorm(y, w, 0.0), rtol=1e-12)
+    np.testing.assert_allclose(oracle.gated_rmsnorm(-y, w, eps), -out, rtol=1e-13)
+    # a huge eps turns it into a plain scaling by weight / sqrt(eps)
+    big = oracle.gated_rmsnorm(y, w, 1e12)
+    np.testing.assert_allclose(big, (w.reshape(H, P) * y) / 1e6, rtol=1e-9)
+    # a permutation of the channels permutes the result (the mean runs over all H*P channels, not per head)
+    perm = rng.permutation(H * P)
+    yp = y.reshape(2, 4, -1)[:, :, perm].reshape(2, 4, H, P)
+    np.testing.assert_allclose(oracle.gated_rmsnorm(yp, w[perm], eps).reshape(2, 4, -1), out.reshape(2, 4, -1)[:, :, perm], rtol=1e-13)
+    # one row does not touch another; padding rows stay NaN
+    y2 = y.copy()
+    y2[1, 3] = np.nan
+    out2 = oracle.gated_rmsnorm(y2, w, eps)
+    assert np.isnan(out2[1, 3]).all()
+    np.testing.assert_array_equal(out2[0], out[0])
+    np.testing.assert_array_equal(out2[1, :3], out[1, :3])
+    with pytest.raises(ValueError):
+        oracle.gated_rmsnorm(y, w[:-1], eps)
