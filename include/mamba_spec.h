@@ -87,6 +87,14 @@ extern "C" {
                                        mamba_spec_commit then makes the other buffer the cache of every sequence with
                                        accept_len == k_draft (nothing is pending for it any more) and records accept_len
                                        as pending for the rest.  mamba_spec_get_selection tells where each cache is.   */
+#define MAMBA_SPEC_FLAG_GATED_RMSNORM 128 /* the normalisation that closes a Mamba-2 block (the hybrid Mamba2 models of
+                                       Sec. 5): every output row is scaled to unit mean square over its H*P channels and
+                                       multiplied by a per-channel weight, after the gate,
+                                         y_t[c] <- io->norm_weight[c] * g_t[c] / sqrt(mean_c(g_t[c]^2) + io->norm_eps),
+                                       g the (gated) output.  The verification kernel writes g in float32 to scratch owned
+                                       by the context (allocated on first use) and a second kernel forms y from it, so the
+                                       output is rounded to the activation dtype once.  Not available without a context
+                                       (mamba_spec_verify_host_static).                                                 */
 
 /* bits of the device status word reported by mamba_spec_status */
 #define MAMBA_SPEC_STATUS_NPREV_CLAMPED 1  /* some n_prev_accepted[b] was outside [0, min(k_max, t_max-k)] */
@@ -131,6 +139,8 @@ typedef struct {
     void *conv_state_k;  /* DEVICE [batch][W-1][H*P] act dtype, output, FLAG_STATE_K only: the conv window
                             after all T_b tokens; must not overlap conv_state                       */
     const float *dt_bias; /* DEVICE [H] float32 ([H*P] with FLAG_MAMBA1), FLAG_DT_SOFTPLUS only; null = no bias */
+    const float *norm_weight; /* DEVICE [H*P] float32, FLAG_GATED_RMSNORM only                                */
+    float norm_eps;       /* FLAG_GATED_RMSNORM only: added to the mean square (>= 0)                                */
 } mamba_spec_io;
 
 /* HOST cfg, HOST out.  Validates the configuration, selects the device and

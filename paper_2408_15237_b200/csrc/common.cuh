@@ -48,6 +48,7 @@ constexpr int kFlagStateK = 8;
 constexpr int kFlagMamba1 = 16;        // interval per channel, A per (channel, state column), D per channel
 constexpr int kFlagDtSoftplus = 32;    // dt arrives raw: softplus(dt + dt_bias) is taken in the kernel
 constexpr int kFlagCommitSelects = 64; // the cache of sequence b is state or state_k as sel[b] says
+constexpr int kFlagGatedRmsnorm = 128; // host side: y goes through float32 scratch and a normalising epilogue kernel
 constexpr int kFlagYNewOnly = 1 << 16; // internal: y holds only the k new rows of each sequence, [batch][k]
 constexpr int kStatusNprevClamped = 1;
 constexpr int kStatusAcceptClamped = 2;

@@ -49,6 +49,12 @@ struct mamba_spec_ctx {
     float *split_state[2] = {nullptr, nullptr};
     void *split_conv[2] = {nullptr, nullptr};
     int32_t *d_zero = nullptr;
+    // FLAG_GATED_RMSNORM: the verification kernel's float32 output rows, read by the normalising kernel; the weight
+    // and eps of the call in progress
+    float *norm_scratch = nullptr;
+    size_t norm_scratch_bytes = 0;
+    const float *norm_w = nullptr;
+    float norm_eps = 0.f;
     cudaStream_t last_stream = nullptr;
     int32_t last_k = -1;
     int64_t launches = 0;
@@ -58,7 +64,8 @@ struct mamba_spec_ctx {
 };
 
 constexpr int kAllFlags = MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K |
-                          MAMBA_SPEC_FLAG_MAMBA1 | MAMBA_SPEC_FLAG_DT_SOFTPLUS | MAMBA_SPEC_FLAG_COMMIT_SELECTS;
+                          MAMBA_SPEC_FLAG_MAMBA1 | MAMBA_SPEC_FLAG_DT_SOFTPLUS | MAMBA_SPEC_FLAG_COMMIT_SELECTS |
+                          MAMBA_SPEC_FLAG_GATED_RMSNORM;
 
 static thread_local std::string g_init_error;
 
@@ -150,6 +157,39 @@ __global__ void commit_kernel(int32_t *n_prev, const int32_t *accept_len, int ba
         a = 0;
     }
     n_prev[b] = a;
+}
+
+// The normalisation that closes a Mamba-2 block, on the float32 rows g the verification kernel left in scratch:
+// y[c] = w[c] g[c] / sqrt(mean_c g[c]^2 + eps) over the C = H*P channels of a token.  One block per token row; rows
+// beyond a sequence's T_b tokens are left alone.
+template <typename out_t>
+__global__ void __launch_bounds__(256) gated_rmsnorm_kernel(out_t *y, const float *g, const float *w, float eps, const int32_t *n_prev,
+                                                            int j_cap, int k, int rows_per_seq, int C, int new_only) {
+    const int row = blockIdx.x, b = row / rows_per_seq, t = row % rows_per_seq;
+    int T = k;
+    if (!new_only) {
+        const int j = n_prev[b];
+        T += j < 0 ? 0 : (j > j_cap ? j_cap : j);
+    }
+    if (t >= T) return;
+    const float *gr = g + (size_t)row * C;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) ss = fmaf(gr[c], gr[c], ss);
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
+    __shared__ float part[8];
+    __shared__ float scale;
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) tot += part[i];
+        scale = 1.0f / sqrtf(tot / (float)C + eps);
+    }
+    __syncthreads();
+    const float r = scale;
+    out_t *yr = y + (size_t)row * C;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) st_act(yr, c, w[c] * gr[c] * r);
 }
 
 }  // namespace
@@ -244,6 +284,14 @@ static int check_and_fill(mamba_spec_ctx *ctx, VerifyParams &p, void *state, voi
         return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "%s: FLAG_STATE_K needs io->state_k and io->conv_state_k", who);
     if ((c.flags & MAMBA_SPEC_FLAG_STATE_K) && (io->state_k == state || io->conv_state_k == conv_state))
         return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "%s: the second snapshot must not alias the cache", who);
+    if (c.flags & MAMBA_SPEC_FLAG_GATED_RMSNORM) {
+        if (!io->norm_weight || !aligned16(io->norm_weight))
+            return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "%s: FLAG_GATED_RMSNORM needs io->norm_weight (16-byte aligned)", who);
+        if (!(io->norm_eps >= 0.f) || io->norm_eps > 3.0e38f)
+            return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "%s: io->norm_eps must be a finite number >= 0", who);
+        ctx->norm_w = io->norm_weight;
+        ctx->norm_eps = io->norm_eps;
+    }
     const void *ptrs[] = {state, conv_state, x, dt, B, C, A, D, io->conv_w, io->conv_b, io->z, io->y,
                           (c.flags & MAMBA_SPEC_FLAG_DT_SOFTPLUS) ? (const void *)io->dt_bias : nullptr,
                           (c.flags & MAMBA_SPEC_FLAG_STATE_K) ? io->state_k : nullptr,
@@ -373,7 +421,7 @@ static SplitPlan plan_split(const VerifyParams &p, const mamba_spec_config &c, i
     return sp;
 }
 
-static int launch(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
+static int launch_blocks(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
     if (ctx->map_cache.size() > 0) {   // (a context that may allocate: the carried state needs scratch)
         const SplitPlan sp = plan_split(p, ctx->cfg, ctx->sm_count, ctx->smem_optin);
         if (sp.split) {
@@ -393,6 +441,42 @@ static int launch(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t strea
         }
     }
     return launch_one(ctx, p, stream, who);
+}
+
+// The whole call: the verification launches and, with FLAG_GATED_RMSNORM, the normalising kernel after them (the
+// verification kernel then writes its output rows in float32 to the context's scratch).
+static int launch(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
+    if (!(p.flags & kFlagGatedRmsnorm)) return launch_blocks(ctx, p, stream, who);
+    const bool new_only = (p.flags & kFlagYNewOnly) != 0;
+    const int rows_per_seq = new_only ? p.k : p.t_max, C = p.H * p.P;
+    if (rows_per_seq < 1) return launch_blocks(ctx, p, stream, who);   // no output rows at all
+    const size_t need = (size_t)p.batch * rows_per_seq * C * sizeof(float);
+    if (ctx->norm_scratch_bytes < need) {
+        if (ctx->norm_scratch) cudaFree(ctx->norm_scratch);   // (synchronises: no launch still uses it)
+        ctx->norm_scratch = nullptr;
+        ctx->norm_scratch_bytes = 0;
+        const cudaError_t e = cudaMalloc(&ctx->norm_scratch, need);
+        if (e != cudaSuccess) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "%s: scratch for the normalised output: %s", who, cudaGetErrorString(e));
+        ctx->norm_scratch_bytes = need;
+    }
+    VerifyParams q = p;
+    q.y = ctx->norm_scratch;
+    q.flags |= kFlagYF32;
+    const int rc = launch_blocks(ctx, q, stream, who);
+    if (rc) return rc;
+    const long long blocks = (long long)p.batch * rows_per_seq;
+    if (blocks > 0x7fffffffLL) return fail(ctx, MAMBA_SPEC_ERR_UNSUPPORTED, "%s: too many output rows for the normalising kernel", who);
+    const bool out_f32 = (p.flags & kFlagYF32) != 0 || ctx->cfg.act_dtype != MAMBA_SPEC_DTYPE_BF16;
+    if (out_f32)
+        gated_rmsnorm_kernel<float><<<(unsigned)blocks, 256, 0, stream>>>((float *)p.y, ctx->norm_scratch, ctx->norm_w, ctx->norm_eps, p.n_prev,
+                                                                           p.j_cap, p.k, rows_per_seq, C, new_only ? 1 : 0);
+    else
+        gated_rmsnorm_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, stream>>>((__nv_bfloat16 *)p.y, ctx->norm_scratch, ctx->norm_w, ctx->norm_eps,
+                                                                                   p.n_prev, p.j_cap, p.k, rows_per_seq, C, new_only ? 1 : 0);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "%s: normalising kernel: %s", who, cudaGetErrorString(e));
+    ctx->launches++;
+    return MAMBA_SPEC_OK;
 }
 
 static int launch_one(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t stream, const char *who) {
@@ -624,6 +708,8 @@ static int verify_host_static_impl(mamba_spec_ctx *tmp, void *state, void *conv_
         return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: configuration rejected (same rules as mamba_spec_init)");
     if (c.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS)
         return fail(tmp, MAMBA_SPEC_ERR_UNSUPPORTED, "verify_host_static: FLAG_COMMIT_SELECTS needs a context");
+    if (c.flags & MAMBA_SPEC_FLAG_GATED_RMSNORM)
+        return fail(tmp, MAMBA_SPEC_ERR_UNSUPPORTED, "verify_host_static: FLAG_GATED_RMSNORM needs a context (scratch for the float32 rows)");
     if (!io) return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: io is null");
     if (!x_host || !dt_host || !B_host || !C_host || !n_prev_host || !io->y)
         return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: a required host pointer is null");
@@ -802,6 +888,7 @@ void mamba_spec_destroy(mamba_spec_ctx *ctx) {
                 if (ctx->split_conv[i]) cudaFree(ctx->split_conv[i]);
             }
             if (ctx->d_zero) cudaFree(ctx->d_zero);
+            if (ctx->norm_scratch) cudaFree(ctx->norm_scratch);
             void *bufs[] = {ctx->d_n_prev, ctx->d_status, ctx->d_sel, ctx->st_x, ctx->st_dt, ctx->st_B, ctx->st_C,
                             ctx->st_z, ctx->st_y, ctx->st_n_prev};
             for (void *b : bufs)

@@ -32,6 +32,7 @@ FLAG_GATE = 1
 FLAG_CONV_SILU = 2
 FLAG_Y_F32 = 4      # outputs in float32 whatever the activation dtype
 FLAG_STATE_K = 8    # second snapshot: the cache after all tokens of the call
+FLAG_GATED_RMSNORM = 128   # the output rows are normalised (unit mean square over H*P channels) and weighted
 
 
 @dataclass(frozen=True)
@@ -201,6 +202,12 @@ class Rounds:
 
 def with_batch(s: Shape, Bt: int) -> Shape:
     return replace(s, Bt=Bt, name=f"{s.name}_bt{Bt}")
+
+
+def norm_params(s: Shape, layer: int = 0):
+    """Weight [H*P] (fp32, around one) and eps of the output normalisation."""
+    g = rng(s.name, layer, "norm")
+    return (1.0 + 0.1 * g.standard_normal(s.H * s.P)).astype(np.float32), 1e-5
 
 
 def m1_params(s: Shape, layer: int = 0):

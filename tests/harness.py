@@ -51,6 +51,10 @@ class Layer:
         self.A, self.D = dev(A, torch.float32), dev(D, torch.float32)
         self.cw, self.cb = dev(cw, torch.float32), dev(cb, torch.float32)
         self.state, self.conv = dev(st, torch.float32), dev(cv, act_dtype(s))
+        self.norm = None
+        if s.flags & synth.FLAG_GATED_RMSNORM:
+            w, eps = synth.norm_params(s, layer)
+            self.norm = (w, eps, dev(w, torch.float32))
 
     def gpu_verify(self, ver, batch, k, y=None, n_prev="given", layer=0):
         s = self.s
@@ -61,8 +65,9 @@ class Layer:
                            dtype=torch.float32 if ver.cfg.flags & synth.FLAG_Y_F32 else ad)
         npv = dev(batch["n_prev"], torch.int32) if n_prev == "given" else None
         z = t["z"] if s.flags & synth.FLAG_GATE else None
+        kw = dict(norm_weight=self.norm[2], norm_eps=self.norm[1]) if self.norm else {}
         ver.verify(self.state, self.conv, t["x"], t["dt"], t["B"], t["C"], self.A, self.D, self.cw, self.cb, z, y,
-                   npv, k, layer=layer)
+                   npv, k, layer=layer, **kw)
         torch.cuda.synchronize()
         return y
 
@@ -71,7 +76,9 @@ class Layer:
         z = batch["z"] if s.flags & synth.FLAG_GATE else None
         y, self.o_state, self.o_conv = oracle.verify(
             self.o_state, self.o_conv, batch["x"], batch["dt"], batch["B"], batch["C"], p["A"], p["D"], p["cw"],
-            p["cb"], z, batch["n_prev"], k, s.flags, threads=threads or oracle.host_threads())
+            p["cb"], z, batch["n_prev"], k, s.flags & (synth.FLAG_GATE | synth.FLAG_CONV_SILU), threads=threads or oracle.host_threads())
+        if self.norm:
+            y = oracle.gated_rmsnorm(y, self.norm[0], self.norm[1])
         return y
 
     def check(self, y_gpu, y_ref, tol, what=""):

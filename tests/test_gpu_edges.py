@@ -218,6 +218,15 @@ def test_argument_errors_are_codes_not_crashes():
     assert binding.lib.mamba_spec_commit(ver.ctx, None, s.Bt, None) == binding.ERR_INVALID_ARG
     torch.cuda.synchronize()
     ver.close()
+    # the normalised output needs its weight and a usable eps
+    ver = h.make_verifier(synth.replace(s, flags=s.flags | synth.FLAG_GATED_RMSNORM), 0)
+    w = torch.ones(s.H * s.P, dtype=torch.float32, device="cuda")
+    assert call(io_over=dict(norm_weight=w.data_ptr(), norm_eps=1e-5)) == 0
+    assert call() == binding.ERR_INVALID_ARG
+    assert call(io_over=dict(norm_weight=w.data_ptr(), norm_eps=-1.0)) == binding.ERR_INVALID_ARG
+    assert call(io_over=dict(norm_weight=w.data_ptr(), norm_eps=float("nan"))) == binding.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    ver.close()
     odd = synth.Shape("unsup", Bt=1, H=3, P=12, N=40, GB=1, GC=3, W=3, k=2, act="fp32")
     v2 = h.make_verifier(odd, STREAM)          # init succeeds; the launch refuses the shape
     lay2 = h.Layer(odd)

@@ -252,3 +252,30 @@ def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects):
                 assert not np.isnan(row).any()
                 assert h.rel_l2(row, y_seq[b, pos]) <= 1e-5, (l, b, pos)
     ver.close()
+
+
+# ------------------------------------------------------------------ gated RMSNorm of the output rows
+NORM_SHAPES = [
+    synth.Shape("norm_small", Bt=3, H=8, P=64, N=128, GB=2, GC=8, W=4, k=4, act="bf16",
+                flags=synth.FLAG_GATE | synth.FLAG_CONV_SILU | synth.FLAG_GATED_RMSNORM),
+    synth.replace(synth.llama8b_layer("norm_llama8b_b4", 4, 4), flags=synth.FLAG_GATE | synth.FLAG_CONV_SILU | synth.FLAG_GATED_RMSNORM),
+    synth.Shape("norm_fp32", Bt=2, H=2, P=16, N=16, GB=1, GC=2, W=4, k=3, act="fp32",
+                flags=synth.FLAG_GATE | synth.FLAG_CONV_SILU | synth.FLAG_GATED_RMSNORM),
+]
+
+
+@pytest.mark.parametrize("kernel", [GENERIC, STREAM])
+@pytest.mark.parametrize("s", NORM_SHAPES, ids=lambda s: s.name)
+@pytest.mark.parametrize("y_f32", [False, True])
+def test_gated_rmsnorm_of_the_output_rows(s, kernel, y_f32):
+    """MAMBA_SPEC_FLAG_GATED_RMSNORM: every output row leaves the call normalised over its H*P channels and weighted
+    (the oracle applies its own gated_rmsnorm to its own outputs); rows beyond T_b stay untouched; the cache is the
+    same as without the flag.  With float32 outputs the bound is 1e-5."""
+    if kernel == STREAM and s.act != "bf16":
+        pytest.skip("the streaming kernel takes bf16 activations")
+    h = H()
+    tol = 1e-5 if (y_f32 or s.act == "fp32") else None
+    worst, name = h.run_rounds(s, 3, kernel=kernel, first_j=2, y_f32=y_f32, tol=tol, final_flush=True)
+    assert ("stream" in name) == (kernel == STREAM)
+    if tol:
+        assert max(worst) <= tol
