@@ -181,6 +181,54 @@ def softplus_dt(dt_raw, bias):
     return np.where(v > 30.0, v, np.log1p(np.exp(np.minimum(v, 30.0))))
 
 
+def conv_rows(rows, window, taps, bias, n_prev, k, silu):
+    """The rolling depthwise causal conv of the Mamba block (Sec. 4.3, footnote) over the token rows of any channel
+    set: ``rows [Bt, Tmax, Ch]`` are the inputs of this call, ``window [Bt, W-1, Ch]`` the last W-1 inputs before
+    them (oldest first), ``taps [Ch, W]`` (tap W-1 multiplies the current token), ``bias [Ch]``.  Returns the
+    outputs ``[Bt, Tmax, Ch]`` (NaN at and beyond ``n_prev[b] + k``) and the window after the first ``n_prev[b]``
+    tokens, i.e. at the newly verified position (unchanged where ``n_prev[b] = 0``)."""
+    rows, window = np.asarray(rows, dtype=np.float64), np.asarray(window, dtype=np.float64)
+    taps, bias = np.asarray(taps, dtype=np.float64), np.asarray(bias, dtype=np.float64)
+    Bt, Tmax, Ch = rows.shape
+    W = taps.shape[1]
+    if window.shape != (Bt, W - 1, Ch) or taps.shape != (Ch, W) or bias.shape != (Ch,):
+        raise ValueError("conv_rows: shapes")
+    out = np.full((Bt, Tmax, Ch), np.nan)
+    win_out = window.copy()
+    for b in range(Bt):
+        j, T = int(n_prev[b]), int(n_prev[b]) + int(k)
+        hist = [window[b, w] for w in range(W - 1)]          # the W-1 inputs before token 0
+        for t in range(T):
+            hist.append(rows[b, t])
+            acc = bias.copy()
+            for w in range(W):
+                acc = acc + taps[:, w] * hist[t + w]          # hist[t + w] is input t - (W-1) + w
+            out[b, t] = acc / (1.0 + np.exp(-acc)) if silu else acc
+            if t == j - 1:
+                for w in range(W - 1):
+                    win_out[b, w] = hist[t + 1 + w]           # the last W-1 inputs up to token j-1
+    return out, win_out
+
+
+def verify_conv_bc(state, conv_state, conv_state_bc, x, dt, Bm, Cm, A, D, conv_w, conv_b, conv_w_bc, conv_b_bc, z, n_prev, k,
+                   flags, threads=1):
+    """The verification call for blocks whose conv runs over x, B and C together (the Mamba-2 block of the hybrid
+    Mamba2 models, Sec. 5): the B and C rows pass through their own depthwise causal conv (channels: the G_B*N
+    columns of B, then the G_C*N columns of C; own taps, bias and rolling window) and the same activation as x
+    before they enter the recurrence.  Returns ``(y, state_out, conv_state_out, conv_state_bc_out)``.
+    Not in the paper's text (parity unpinned by the paper); the conv itself is the one of Sec. 4.3."""
+    Bm, Cm = np.asarray(Bm, dtype=np.float64), np.asarray(Cm, dtype=np.float64)
+    Bt, Tmax, GB, N = Bm.shape
+    GC = Cm.shape[2]
+    rows = np.concatenate([Bm.reshape(Bt, Tmax, GB * N), Cm.reshape(Bt, Tmax, GC * N)], axis=2)
+    out, win = conv_rows(rows, conv_state_bc, conv_w_bc, conv_b_bc, n_prev, k, bool(flags & 2))
+    out = np.nan_to_num(out)     # rows beyond T_b are never read by the recurrence
+    Bc = out[:, :, :GB * N].reshape(Bt, Tmax, GB, N)
+    Cc = out[:, :, GB * N:].reshape(Bt, Tmax, GC, N)
+    y, s_out, c_out = verify(state, conv_state, x, dt, Bc, Cc, A, D, conv_w, conv_b, z, n_prev, k, flags, threads=threads)
+    return y, s_out, c_out, win
+
+
 def gated_rmsnorm(y, weight, eps):
     """The output normalisation of the Mamba-2 blocks that the hybrid Mamba2 models (Sec. 5) are made of: with
     ``y`` the gated output of the verification call, ``[..., H, P]``, every token row is scaled to unit mean

@@ -481,3 +481,91 @@ def test_gated_rmsnorm_against_its_definition_and_invariants():
     np.testing.assert_array_equal(out2[1, :3], out[1, :3])
     with pytest.raises(ValueError):
         oracle.gated_rmsnorm(y, w[:-1], eps)
+
+
+# --------------------------------------------------------------------------- conv over the B and C channels
+def bc_problem(seed, **kw):
+    q = small_problem(seed, **kw)
+    g = np.random.default_rng(seed + 1000)
+    Bt, T, GB, N = q["B"].shape
+    GC, W = q["C"].shape[2], q["cw"].shape[1]
+    ch = (GB + GC) * N
+    q.update(conv_bc=0.5 * g.standard_normal((Bt, W - 1, ch)), cw_bc=g.standard_normal((ch, W)) / 2, cb_bc=0.1 * g.standard_normal(ch))
+    return q
+
+
+def run_verify_bc(q, n_prev, k, flags, **over):
+    a = dict(q, **over)
+    return oracle.verify_conv_bc(a["state"], a["conv"], a["conv_bc"], a["x"], a["dt"], a["B"], a["C"], a["A"], a["D"], a["cw"], a["cb"],
+                                 a["cw_bc"], a["cb_bc"], a["z"], n_prev, k, flags)
+
+
+def test_conv_rows_against_numpy_correlate_and_its_special_kernels():
+    g = np.random.default_rng(5)
+    Bt, T, Ch, W = 2, 9, 6, 4
+    rows, window = g.standard_normal((Bt, T, Ch)), g.standard_normal((Bt, W - 1, Ch))
+    taps, bias = g.standard_normal((Ch, W)), g.standard_normal(Ch)
+    n_prev = np.array([4, 0], dtype=np.int32)
+    out, win = oracle.conv_rows(rows, window, taps, bias, n_prev, 5, False)
+    for b in range(Bt):
+        Tb = n_prev[b] + 5
+        for c in range(Ch):
+            hist = np.concatenate([window[b, :, c], rows[b, :, c]])
+            full = np.correlate(hist, taps[c], mode="valid") + bias[c]     # tap W-1 on the current token
+            np.testing.assert_allclose(out[b, :Tb, c], full[:Tb], rtol=1e-13, atol=1e-14)
+        assert np.isnan(out[b, Tb:]).all()
+        hist = np.concatenate([window[b], rows[b, :n_prev[b]]])
+        np.testing.assert_array_equal(win[b], hist[-(W - 1):])              # window at the verified position
+    silu, _ = oracle.conv_rows(rows, window, taps, bias, n_prev, 5, True)
+    np.testing.assert_allclose(silu[0, :9], out[0, :9] / (1 + np.exp(-out[0, :9])), rtol=1e-13)
+    delta = np.zeros((Ch, W))
+    delta[:, -1] = 1.0
+    ident, _ = oracle.conv_rows(rows, window, delta, np.zeros(Ch), n_prev, 5, False)
+    np.testing.assert_array_equal(ident[0, :9], rows[0, :9])
+    oldest = np.zeros((Ch, W))
+    oldest[:, 0] = 1.0
+    delayed, _ = oracle.conv_rows(rows, window, oldest, np.zeros(Ch), n_prev, 5, False)
+    np.testing.assert_array_equal(delayed[0, 3:9], rows[0, 0:6])
+    np.testing.assert_array_equal(delayed[0, 0:3], window[0])
+
+
+def test_conv_over_b_and_c_reduces_to_the_plain_call_and_chains_like_it():
+    q = bc_problem(31)
+    n_prev = np.array([0, 2, 3], dtype=np.int32)
+    # identity taps and no activation: B and C pass through unchanged, the call is the pinned one
+    ch, W = q["cw_bc"].shape
+    delta = np.zeros((ch, W))
+    delta[:, -1] = 1.0
+    y0, s0, c0 = run_verify(q, n_prev, 3, GATE)
+    y1, s1, c1, w1 = run_verify_bc(q, n_prev, 3, GATE, cw_bc=delta, cb_bc=np.zeros(ch))
+    np.testing.assert_array_equal(np.nan_to_num(y1), np.nan_to_num(y0))
+    np.testing.assert_array_equal(s1, s0)
+    np.testing.assert_array_equal(c1, c0)
+    # with real taps: the recurrence sees exactly conv_rows' outputs (B channels first, then C)
+    Bt, T, GB, N = q["B"].shape
+    GC = q["C"].shape[2]
+    rows = np.concatenate([q["B"].reshape(Bt, T, -1), q["C"].reshape(Bt, T, -1)], axis=2)
+    out, win = oracle.conv_rows(rows, q["conv_bc"], q["cw_bc"], q["cb_bc"], n_prev, 3, True)
+    out = np.nan_to_num(out)
+    y2, s2, c2, w2 = run_verify_bc(q, n_prev, 3, GATE | CSILU)
+    y3, s3, c3 = run_verify(q, n_prev, 3, GATE | CSILU, B=out[:, :, :GB * N].reshape(Bt, T, GB, N), C=out[:, :, GB * N:].reshape(Bt, T, GC, N))
+    np.testing.assert_array_equal(np.nan_to_num(y2), np.nan_to_num(y3))
+    np.testing.assert_array_equal(s2, s3)
+    np.testing.assert_array_equal(w2, win)
+    # a call that replays j tokens and drafts k equals a call over the j tokens followed by one over the k drafts
+    # from the caches the first one left (state, both conv windows)
+    ya, sa, ca, wa = run_verify_bc(q, n_prev, 3, GATE | CSILU)
+    zero = np.zeros(3, dtype=np.int32)
+    for b in range(3):
+        j = int(n_prev[b])
+        sl = slice(b, b + 1)
+        qa = {k_: (v[sl] if k_ in ("state", "conv", "conv_bc", "x", "z", "dt", "B", "C") else v) for k_, v in q.items()}
+        nb = np.array([j], dtype=np.int32)
+        _, s_first, c_first, w_first = run_verify_bc(qa, nb, 0, GATE | CSILU)
+        np.testing.assert_allclose(s_first, sa[sl], rtol=1e-13, atol=1e-15)
+        np.testing.assert_array_equal(w_first, wa[sl])
+        qb = dict(qa, state=s_first, conv=c_first, conv_bc=w_first)
+        for name in ("x", "z", "dt", "B", "C"):
+            qb[name] = np.concatenate([qa[name][:, j:], np.zeros_like(qa[name][:, :j])], axis=1)
+        y_second, _, _, _ = run_verify_bc(qb, np.zeros(1, dtype=np.int32), 3, GATE | CSILU)
+        np.testing.assert_allclose(y_second[0, :3], ya[b, j:j + 3], rtol=1e-12, atol=1e-13)
