@@ -95,6 +95,13 @@ extern "C" {
                                        by the context (allocated on first use) and a second kernel forms y from it, so the
                                        output is rounded to the activation dtype once.  Not available without a context
                                        (mamba_spec_verify_host_static).                                                 */
+#define MAMBA_SPEC_FLAG_CONV_BC 256 /* the conv of a Mamba-2 block runs over x, B and C together: the B and C rows pass through
+                                       a depthwise causal conv of their own (channels: the G_B*N columns of B, then the
+                                       G_C*N columns of C; taps io->conv_w_bc, bias io->conv_b_bc, rolling window
+                                       io->conv_state_bc, cached at the verified position like conv_state) and the same
+                                       activation as x before they enter the recurrence.  Generic kernel only (the
+                                       streaming kernel refuses the flag); not with FLAG_STATE_K.  The conv's float32
+                                       outputs live in scratch owned by the context.                                   */
 
 /* bits of the device status word reported by mamba_spec_status */
 #define MAMBA_SPEC_STATUS_NPREV_CLAMPED 1  /* some n_prev_accepted[b] was outside [0, min(k_max, t_max-k)] */
@@ -141,6 +148,10 @@ typedef struct {
     const float *dt_bias; /* DEVICE [H] float32 ([H*P] with FLAG_MAMBA1), FLAG_DT_SOFTPLUS only; null = no bias */
     const float *norm_weight; /* DEVICE [H*P] float32, FLAG_GATED_RMSNORM only                                */
     float norm_eps;       /* FLAG_GATED_RMSNORM only: added to the mean square (>= 0)                                */
+    void *conv_state_bc;  /* DEVICE [batch][W-1][(G_B+G_C)*N] act dtype, in/out, FLAG_CONV_BC only: the last W-1 B and C
+                             rows at the cached position, oldest first                                            */
+    const float *conv_w_bc; /* DEVICE [(G_B+G_C)*N][W] float32, FLAG_CONV_BC only; tap W-1 multiplies the current token    */
+    const float *conv_b_bc; /* DEVICE [(G_B+G_C)*N] float32, FLAG_CONV_BC only                                            */
 } mamba_spec_io;
 
 /* HOST cfg, HOST out.  Validates the configuration, selects the device and

@@ -24,7 +24,7 @@ lib = ctypes.CDLL(str(_LIB_PATH))
 OK = 0
 DTYPE_F32, DTYPE_BF16 = 0, 1
 FLAG_GATE, FLAG_CONV_SILU, FLAG_Y_F32, FLAG_STATE_K = 1, 2, 4, 8
-FLAG_MAMBA1, FLAG_DT_SOFTPLUS, FLAG_COMMIT_SELECTS, FLAG_GATED_RMSNORM = 16, 32, 64, 128
+FLAG_MAMBA1, FLAG_DT_SOFTPLUS, FLAG_COMMIT_SELECTS, FLAG_GATED_RMSNORM, FLAG_CONV_BC = 16, 32, 64, 128, 256
 STATUS_NPREV_CLAMPED, STATUS_ACCEPT_CLAMPED, STATUS_COPY_TIMEOUT = 1, 2, 4
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_STREAM = 0, 1, 2
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_MISALIGNED, ERR_UNSUPPORTED, ERR_CUDA, ERR_NOT_INIT = -1, -2, -3, -4, -5, -6
@@ -41,7 +41,8 @@ class IO(ctypes.Structure):
                 ("y", ctypes.c_void_p), ("batch", ctypes.c_int32), ("layer", ctypes.c_int32),
                 ("t_max", ctypes.c_int32), ("stream", ctypes.c_void_p), ("state_k", ctypes.c_void_p),
                 ("conv_state_k", ctypes.c_void_p), ("dt_bias", ctypes.c_void_p), ("norm_weight", ctypes.c_void_p),
-                ("norm_eps", ctypes.c_float)]
+                ("norm_eps", ctypes.c_float), ("conv_state_bc", ctypes.c_void_p), ("conv_w_bc", ctypes.c_void_p),
+                ("conv_b_bc", ctypes.c_void_p)]
 
 
 _vp, _i32 = ctypes.c_void_p, ctypes.c_int32
@@ -198,7 +199,7 @@ class Verifier:
             pass
 
     def _io(self, conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k=None, conv_state_k=None, dt_bias=None,
-            norm_weight=None, norm_eps=0.0):
+            norm_weight=None, norm_eps=0.0, conv_bc=None):
         if stream is None:
             stream = torch.cuda.current_stream().cuda_stream
         if norm_weight is not None:
@@ -207,10 +208,23 @@ class Verifier:
                     not norm_weight.is_contiguous():
                 raise ValueError(f"norm_weight: want contiguous CUDA torch.float32 ({chan},)")
         return IO(_ptr(conv_w), _ptr(conv_b), _ptr(z), _ptr(y), batch, layer, t_max, stream, _ptr(state_k),
-                  _ptr(conv_state_k), _ptr(dt_bias), _ptr(norm_weight), float(norm_eps))
+                  _ptr(conv_state_k), _ptr(dt_bias), _ptr(norm_weight), float(norm_eps), *self._conv_bc(conv_bc, batch))
+
+    def _conv_bc(self, conv_bc, batch):
+        """(window, taps, bias) of the conv over the B and C channels as three pointers, shapes checked."""
+        if conv_bc is None:
+            return None, None, None
+        c = self.cfg
+        ch = (c.n_groups_b + c.n_groups_c) * c.d_state
+        window, taps, bias = conv_bc
+        for name, t, dtype, shape in (("conv_state_bc", window, self.act_dtype, (batch, c.conv_width - 1, ch)),
+                                      ("conv_w_bc", taps, torch.float32, (ch, c.conv_width)), ("conv_b_bc", bias, torch.float32, (ch,))):
+            if not t.is_cuda or t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
+                raise ValueError(f"{name}: want contiguous CUDA {dtype} {shape}, got {t.dtype} {tuple(t.shape)}")
+        return _ptr(window), _ptr(taps), _ptr(bias)
 
     def verify(self, state, conv_state, x, dt, B, C, A, D, conv_w, conv_b, z, y, n_prev, k, layer=0, stream=None,
-               state_k=None, conv_state_k=None, dt_bias=None, norm_weight=None, norm_eps=0.0):
+               state_k=None, conv_state_k=None, dt_bias=None, norm_weight=None, norm_eps=0.0, conv_bc=None):
         c = self.cfg
         batch, t_max = x.shape[0], x.shape[1]
         m1 = bool(c.flags & FLAG_MAMBA1)
@@ -246,7 +260,7 @@ class Verifier:
                 t, dtype, shape = want[name]
                 if not t.is_cuda or t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
                     raise ValueError(f"{name}: want contiguous CUDA {dtype} {shape}")
-        io = self._io(conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k, conv_state_k, dt_bias, norm_weight, norm_eps)
+        io = self._io(conv_w, conv_b, z, y, batch, layer, t_max, stream, state_k, conv_state_k, dt_bias, norm_weight, norm_eps, conv_bc)
         mamba_spec_verify(self.ctx, state, conv_state, x, dt, B, C, A, D, n_prev, k, io)
 
     def verify_new(self, state, conv_state, x_new, dt_new, B_new, C_new, A, D, conv_w, conv_b, z_new, y_new, k, layer=0,

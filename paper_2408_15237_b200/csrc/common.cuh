@@ -48,6 +48,7 @@ constexpr int kFlagStateK = 8;
 constexpr int kFlagMamba1 = 16;        // interval per channel, A per (channel, state column), D per channel
 constexpr int kFlagDtSoftplus = 32;    // dt arrives raw: softplus(dt + dt_bias) is taken in the kernel
 constexpr int kFlagCommitSelects = 64; // the cache of sequence b is state or state_k as sel[b] says
+constexpr int kFlagConvBC = 256;       // B and C pass through a depthwise conv of their own first (generic kernel only)
 constexpr int kFlagGatedRmsnorm = 128; // host side: y goes through float32 scratch and a normalising epilogue kernel
 constexpr int kFlagYNewOnly = 1 << 16; // internal: y holds only the k new rows of each sequence, [batch][k]
 constexpr int kStatusNprevClamped = 1;
@@ -85,9 +86,25 @@ __device__ __forceinline__ int load_n_prev(const VerifyParams &p, int b) {
     j -= p.n_prev_done;
     return j < 0 ? 0 : (j > p.j_cap ? p.j_cap : j);
 }
+// The same value without the report (for a second kernel that reads the same entry).
+__device__ __forceinline__ int peek_n_prev(const VerifyParams &p, int b) {
+    int j = p.n_prev[b];
+    const int full = p.n_prev_full ? p.n_prev_full : p.j_cap;
+    j = j < 0 ? 0 : (j > full ? full : j);
+    j -= p.n_prev_done;
+    return j < 0 ? 0 : (j > p.j_cap ? p.j_cap : j);
+}
 
 // Launchers (defined in verify_generic.cu / verify_stream.cu).  Return cudaGetLastError().
-cudaError_t launch_verify_generic(const VerifyParams &p, bool bf16, cudaStream_t stream);
+// FLAG_CONV_BC: what the conv over the B and C channels needs beside VerifyParams.  Channel c of the
+// (GB + GC) * N channels is column c of B for c < GB * N, else column c - GB * N of C.
+struct ConvBC {
+    void *window;        // [batch][W-1][(GB+GC)*N] act dtype, in/out: the last W-1 B and C rows at the cached position
+    const float *taps;   // [(GB+GC)*N][W]
+    const float *bias;   // [(GB+GC)*N]
+    float *out;          // scratch, float32: the conv's outputs laid out like B, [batch][t_max][GB][N], then like C
+};
+cudaError_t launch_verify_generic(const VerifyParams &p, bool bf16, cudaStream_t stream, const ConvBC *bc = nullptr);
 
 // Shared-memory plan of the streaming kernel: ring depths and byte offsets (all multiples of 16).
 struct StreamLayout {

@@ -55,6 +55,10 @@ struct mamba_spec_ctx {
     size_t norm_scratch_bytes = 0;
     const float *norm_w = nullptr;
     float norm_eps = 0.f;
+    // FLAG_CONV_BC: the float32 outputs of the conv over the B and C rows, and the call's window, taps and bias
+    float *bc_scratch = nullptr;
+    size_t bc_scratch_bytes = 0;
+    ConvBC bc = {nullptr, nullptr, nullptr, nullptr};
     cudaStream_t last_stream = nullptr;
     int32_t last_k = -1;
     int64_t launches = 0;
@@ -65,7 +69,7 @@ struct mamba_spec_ctx {
 
 constexpr int kAllFlags = MAMBA_SPEC_FLAG_GATE | MAMBA_SPEC_FLAG_CONV_SILU | MAMBA_SPEC_FLAG_Y_F32 | MAMBA_SPEC_FLAG_STATE_K |
                           MAMBA_SPEC_FLAG_MAMBA1 | MAMBA_SPEC_FLAG_DT_SOFTPLUS | MAMBA_SPEC_FLAG_COMMIT_SELECTS |
-                          MAMBA_SPEC_FLAG_GATED_RMSNORM;
+                          MAMBA_SPEC_FLAG_GATED_RMSNORM | MAMBA_SPEC_FLAG_CONV_BC;
 
 static thread_local std::string g_init_error;
 
@@ -220,6 +224,10 @@ int mamba_spec_init(const mamba_spec_config *cfg, mamba_spec_ctx **out) {
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: unknown kernel_select %d", c.kernel_select);
     if ((c.flags & MAMBA_SPEC_FLAG_COMMIT_SELECTS) && !(c.flags & MAMBA_SPEC_FLAG_STATE_K))
         return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: FLAG_COMMIT_SELECTS needs FLAG_STATE_K");
+    if ((c.flags & MAMBA_SPEC_FLAG_CONV_BC) && (c.flags & MAMBA_SPEC_FLAG_STATE_K))
+        return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: FLAG_CONV_BC keeps one window of B and C rows: not with FLAG_STATE_K");
+    if ((c.flags & MAMBA_SPEC_FLAG_CONV_BC) && c.kernel_select == MAMBA_SPEC_KERNEL_STREAM)
+        return fail(nullptr, MAMBA_SPEC_ERR_INVALID_ARG, "init: FLAG_CONV_BC runs in the generic kernel");
     // conv_state rows and token rows must keep 16-byte alignment per (sequence, row)
     if ((size_t)c.n_heads * c.head_dim * act_bytes(c) % 16)
         return fail(nullptr, MAMBA_SPEC_ERR_BAD_SHAPE, "init: H*P*sizeof(act) must be a multiple of 16 bytes");
@@ -291,6 +299,15 @@ static int check_and_fill(mamba_spec_ctx *ctx, VerifyParams &p, void *state, voi
             return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "%s: io->norm_eps must be a finite number >= 0", who);
         ctx->norm_w = io->norm_weight;
         ctx->norm_eps = io->norm_eps;
+    }
+    if (c.flags & MAMBA_SPEC_FLAG_CONV_BC) {
+        if (!io->conv_w_bc || !io->conv_b_bc || (c.conv_width > 1 && !io->conv_state_bc))
+            return fail(ctx, MAMBA_SPEC_ERR_INVALID_ARG, "%s: FLAG_CONV_BC needs io->conv_state_bc, io->conv_w_bc and io->conv_b_bc", who);
+        if (!aligned16(io->conv_w_bc) || !aligned16(io->conv_b_bc) || !aligned16(io->conv_state_bc))
+            return fail(ctx, MAMBA_SPEC_ERR_MISALIGNED, "%s: a tensor of the conv over B and C is not 16-byte aligned", who);
+        ctx->bc.window = io->conv_state_bc;
+        ctx->bc.taps = io->conv_w_bc;
+        ctx->bc.bias = io->conv_b_bc;
     }
     const void *ptrs[] = {state, conv_state, x, dt, B, C, A, D, io->conv_w, io->conv_b, io->z, io->y,
                           (c.flags & MAMBA_SPEC_FLAG_DT_SOFTPLUS) ? (const void *)io->dt_bias : nullptr,
@@ -518,7 +535,24 @@ static int launch_one(mamba_spec_ctx *ctx, const VerifyParams &p, cudaStream_t s
         if (c.kernel_select == MAMBA_SPEC_KERNEL_STREAM)
             return fail(ctx, MAMBA_SPEC_ERR_UNSUPPORTED, "%s: streaming kernel does not take this shape (%s)", who, plan.name);
     }
-    e = launch_verify_generic(p, bf16, stream);
+    const ConvBC *bcp = nullptr;
+    if (p.flags & kFlagConvBC) {   // the conv over the B and C rows runs first, into scratch
+        const size_t need = (size_t)p.batch * p.t_max * (p.GB + p.GC) * p.N * sizeof(float);
+        if (ctx->bc_scratch_bytes < need) {
+            if (ctx->map_cache.empty())
+                return fail(ctx, MAMBA_SPEC_ERR_UNSUPPORTED, "%s: FLAG_CONV_BC needs a context (scratch for the conv's outputs)", who);
+            if (ctx->bc_scratch) cudaFree(ctx->bc_scratch);   // (synchronises: no launch still uses it)
+            ctx->bc_scratch = nullptr;
+            ctx->bc_scratch_bytes = 0;
+            e = cudaMalloc(&ctx->bc_scratch, need);
+            if (e != cudaSuccess) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "%s: scratch for the conv over B and C: %s", who, cudaGetErrorString(e));
+            ctx->bc_scratch_bytes = need;
+        }
+        ctx->bc.out = ctx->bc_scratch;
+        bcp = &ctx->bc;
+        ctx->launches++;
+    }
+    e = launch_verify_generic(p, bf16, stream, bcp);
     if (e != cudaSuccess) return fail(ctx, MAMBA_SPEC_ERR_CUDA, "%s: generic launch: %s", who, cudaGetErrorString(e));
     snprintf(ctx->last_kernel, sizeof ctx->last_kernel, "generic");
     ctx->launches++;
@@ -710,6 +744,8 @@ static int verify_host_static_impl(mamba_spec_ctx *tmp, void *state, void *conv_
         return fail(tmp, MAMBA_SPEC_ERR_UNSUPPORTED, "verify_host_static: FLAG_COMMIT_SELECTS needs a context");
     if (c.flags & MAMBA_SPEC_FLAG_GATED_RMSNORM)
         return fail(tmp, MAMBA_SPEC_ERR_UNSUPPORTED, "verify_host_static: FLAG_GATED_RMSNORM needs a context (scratch for the float32 rows)");
+    if (c.flags & MAMBA_SPEC_FLAG_CONV_BC)
+        return fail(tmp, MAMBA_SPEC_ERR_UNSUPPORTED, "verify_host_static: FLAG_CONV_BC needs a context (scratch for the conv's outputs)");
     if (!io) return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: io is null");
     if (!x_host || !dt_host || !B_host || !C_host || !n_prev_host || !io->y)
         return fail(tmp, MAMBA_SPEC_ERR_INVALID_ARG, "verify_host_static: a required host pointer is null");
@@ -889,6 +925,7 @@ void mamba_spec_destroy(mamba_spec_ctx *ctx) {
             }
             if (ctx->d_zero) cudaFree(ctx->d_zero);
             if (ctx->norm_scratch) cudaFree(ctx->norm_scratch);
+            if (ctx->bc_scratch) cudaFree(ctx->bc_scratch);
             void *bufs[] = {ctx->d_n_prev, ctx->d_status, ctx->d_sel, ctx->st_x, ctx->st_dt, ctx->st_B, ctx->st_C,
                             ctx->st_z, ctx->st_y, ctx->st_n_prev};
             for (void *b : bufs)

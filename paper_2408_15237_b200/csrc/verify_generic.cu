@@ -21,7 +21,54 @@
 
 namespace mspec {
 
-template <typename act_t, bool M1>
+// FLAG_CONV_BC: the rolling depthwise causal conv (Sec. 4.3, footnote) over the B and C rows, one thread per
+// (sequence, channel), ahead of the recurrence: outputs in float32 to scratch laid out like B and C
+// ([batch][t_max][GB][N] followed by [batch][t_max][GC][N]), the window at the verified position written back.
+template <typename act_t>
+__global__ void __launch_bounds__(128) conv_bc_kernel(const VerifyParams p, const ConvBC bc) {
+    const int chB = p.GB * p.N, chC = p.GC * p.N, ch = chB + chC;
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)p.batch * ch) return;
+    const int b = (int)(i / ch), c = (int)(i % ch);
+    const int j = peek_n_prev(p, b), T = j + p.k, W = p.W;
+    const bool isB = c < chB;
+    const act_t *src = isB ? (const act_t *)p.B : (const act_t *)p.C;
+    const int cc = isB ? c : c - chB, cw = isB ? chB : chC;
+    float *dst = bc.out + (isB ? 0 : (size_t)p.batch * p.t_max * chB);
+    act_t *window = (act_t *)bc.window;
+    float win[kMaxConvWidth - 1], tap[kMaxConvWidth];
+#pragma unroll
+    for (int w = 0; w < kMaxConvWidth - 1; ++w) win[w] = (w < W - 1) ? ld_act(window, ((size_t)b * (W - 1) + w) * ch + c) : 0.f;
+#pragma unroll
+    for (int w = 0; w < kMaxConvWidth; ++w) tap[w] = (w < W) ? bc.taps[(size_t)c * W + w] : 0.f;
+    const float bias = bc.bias[c];
+    const int row_first = first_row(p, b);
+    for (int t = 0; t < T; ++t) {
+        const size_t bt = (size_t)b * p.t_max + row_first + t;
+        const float in = ld_act(src, bt * cw + cc);
+        float acc = bias;
+#pragma unroll
+        for (int w = 0; w < kMaxConvWidth - 1; ++w)
+            if (w < W - 1) acc = fmaf(tap[w], win[w], acc);
+#pragma unroll
+        for (int w = 0; w < kMaxConvWidth; ++w)
+            if (w == W - 1) acc = fmaf(tap[w], in, acc);
+        dst[bt * cw + cc] = (p.flags & kFlagConvSilu) ? silu_f(acc) : acc;
+#pragma unroll
+        for (int w = 0; w < kMaxConvWidth - 2; ++w)
+            if (w < W - 2) win[w] = win[w + 1];
+#pragma unroll
+        for (int w = 0; w < kMaxConvWidth - 1; ++w)
+            if (w == W - 2) win[w] = in;
+        if (t == j - 1) {
+#pragma unroll
+            for (int w = 0; w < kMaxConvWidth - 1; ++w)
+                if (w < W - 1) st_act(window, ((size_t)b * (W - 1) + w) * ch + c, win[w]);
+        }
+    }
+}
+
+template <typename act_t, bool M1, typename bc_t>
 __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams p) {
     const int lane = threadIdx.x & 31;
     const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -36,8 +83,8 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
 
     const int N = p.N, W = p.W, H = p.H, P = p.P;
     const int Cch = H * P, c = h * P + pr;
-    const act_t *x = (const act_t *)p.x, *dt = (const act_t *)p.dt, *Bm = (const act_t *)p.B,
-                *Cm = (const act_t *)p.C, *z = (const act_t *)p.z;
+    const act_t *x = (const act_t *)p.x, *dt = (const act_t *)p.dt, *z = (const act_t *)p.z;
+    const bc_t *Bm = (const bc_t *)p.B, *Cm = (const bc_t *)p.C;   // (float32 after their own conv, FLAG_CONV_BC)
     act_t *y = (act_t *)p.y;
     // commit-selects mode: this sequence's cache is the second pair of buffers when sel says so; the state
     // at the verified position goes back to where the cache is, the state after all tokens to the other pair
@@ -89,7 +136,7 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
         float dtv = ld_act(dt, M1 ? bt * Cch + c : bt * H + h);
         if (sp) dtv = softplus_f(dtv + dtb);
         const float a = M1 ? 0.f : expf(dtv * A_h), u = dtv * xc;
-        const act_t *Bv = Bm + (bt * p.GB + gB) * N, *Cv = Cm + (bt * p.GC + gC) * N;
+        const bc_t *Bv = Bm + (bt * p.GB + gB) * N, *Cv = Cm + (bt * p.GC + gC) * N;
         float part = 0.f;
 #pragma unroll
         for (int i = 0; i < kRegs; ++i) {
@@ -136,16 +183,34 @@ __global__ void __launch_bounds__(128) verify_generic_kernel(const VerifyParams 
     }
 }
 
-cudaError_t launch_verify_generic(const VerifyParams &p, bool bf16, cudaStream_t stream) {
+cudaError_t launch_verify_generic(const VerifyParams &p, bool bf16, cudaStream_t stream, const ConvBC *bc) {
     const long long rows = (long long)p.batch * p.H * p.P;
     const int warps_per_block = 4;
     const long long blocks = (rows + warps_per_block - 1) / warps_per_block;
     if (blocks <= 0 || blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     const bool m1 = (p.flags & kFlagMamba1) != 0;
-    if (bf16 && m1) verify_generic_kernel<__nv_bfloat16, true><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
-    else if (bf16) verify_generic_kernel<__nv_bfloat16, false><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
-    else if (m1) verify_generic_kernel<float, true><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
-    else verify_generic_kernel<float, false><<<(unsigned)blocks, warps_per_block * 32, 0, stream>>>(p);
+    const unsigned nb = (unsigned)blocks, nt = warps_per_block * 32;
+    if (bc != nullptr) {
+        // the conv over the B and C rows first; the recurrence then reads its float32 outputs in their place
+        const long long items = (long long)p.batch * (p.GB + p.GC) * p.N, cblocks = (items + 127) / 128;
+        if (cblocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+        if (bf16) conv_bc_kernel<__nv_bfloat16><<<(unsigned)cblocks, 128, 0, stream>>>(p, *bc);
+        else conv_bc_kernel<float><<<(unsigned)cblocks, 128, 0, stream>>>(p, *bc);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        VerifyParams q = p;
+        q.B = bc->out;
+        q.C = bc->out + (size_t)p.batch * p.t_max * p.GB * p.N;
+        if (bf16 && m1) verify_generic_kernel<__nv_bfloat16, true, float><<<nb, nt, 0, stream>>>(q);
+        else if (bf16) verify_generic_kernel<__nv_bfloat16, false, float><<<nb, nt, 0, stream>>>(q);
+        else if (m1) verify_generic_kernel<float, true, float><<<nb, nt, 0, stream>>>(q);
+        else verify_generic_kernel<float, false, float><<<nb, nt, 0, stream>>>(q);
+        return cudaGetLastError();
+    }
+    if (bf16 && m1) verify_generic_kernel<__nv_bfloat16, true, __nv_bfloat16><<<nb, nt, 0, stream>>>(p);
+    else if (bf16) verify_generic_kernel<__nv_bfloat16, false, __nv_bfloat16><<<nb, nt, 0, stream>>>(p);
+    else if (m1) verify_generic_kernel<float, true, float><<<nb, nt, 0, stream>>>(p);
+    else verify_generic_kernel<float, false, float><<<nb, nt, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

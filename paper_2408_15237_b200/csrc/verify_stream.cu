@@ -952,6 +952,7 @@ StreamPlan plan_verify_stream(const VerifyParams &p, bool bf16, int sm_count, si
     };
     if (!bf16) return reject("activations are not bf16");
     if (p.flags & kFlagMamba1) return reject("the Mamba-1 parameterisation runs in the generic kernel");
+    if (p.flags & kFlagConvBC) return reject("the conv over the B and C channels runs with the generic kernel");
     if (p.W != kW) return reject("conv width is not 4");
     if (p.N != 64 && p.N != 128) return reject("state dim is not 64 or 128");
     if (p.P % 32) return reject("head dim is not a multiple of 32");

@@ -33,6 +33,7 @@ FLAG_CONV_SILU = 2
 FLAG_Y_F32 = 4      # outputs in float32 whatever the activation dtype
 FLAG_STATE_K = 8    # second snapshot: the cache after all tokens of the call
 FLAG_GATED_RMSNORM = 128   # the output rows are normalised (unit mean square over H*P channels) and weighted
+FLAG_CONV_BC = 256         # the B and C rows pass through a depthwise conv of their own before the recurrence
 
 
 @dataclass(frozen=True)
@@ -202,6 +203,17 @@ class Rounds:
 
 def with_batch(s: Shape, Bt: int) -> Shape:
     return replace(s, Bt=Bt, name=f"{s.name}_bt{Bt}")
+
+
+def conv_bc_params(s: Shape, layer: int = 0):
+    """Taps [(GB+GC)*N, W], bias [(GB+GC)*N] (fp32) and the initial window [Bt, W-1, (GB+GC)*N] (activation precision)
+    of the conv over the B and C channels."""
+    g = rng(s.name, layer, "conv_bc")
+    ch = (s.GB + s.GC) * s.N
+    taps = (g.standard_normal((ch, s.W)) / np.sqrt(s.W)).astype(np.float32)
+    bias = (0.1 * g.standard_normal(ch)).astype(np.float32)
+    window = to_act((0.1 * g.standard_normal((s.Bt, s.W - 1, ch))).astype(np.float32), s.act)
+    return taps, bias, window
 
 
 def norm_params(s: Shape, layer: int = 0):

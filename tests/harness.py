@@ -51,6 +51,11 @@ class Layer:
         self.A, self.D = dev(A, torch.float32), dev(D, torch.float32)
         self.cw, self.cb = dev(cw, torch.float32), dev(cb, torch.float32)
         self.state, self.conv = dev(st, torch.float32), dev(cv, act_dtype(s))
+        self.bc = None
+        if s.flags & synth.FLAG_CONV_BC:
+            taps, bias, window = synth.conv_bc_params(s, layer)
+            self.bc = dict(taps=taps, bias=bias, o_window=window.astype(np.float64),
+                           dev=(dev(window, act_dtype(s)), dev(taps, torch.float32), dev(bias, torch.float32)))
         self.norm = None
         if s.flags & synth.FLAG_GATED_RMSNORM:
             w, eps = synth.norm_params(s, layer)
@@ -66,6 +71,8 @@ class Layer:
         npv = dev(batch["n_prev"], torch.int32) if n_prev == "given" else None
         z = t["z"] if s.flags & synth.FLAG_GATE else None
         kw = dict(norm_weight=self.norm[2], norm_eps=self.norm[1]) if self.norm else {}
+        if self.bc:
+            kw["conv_bc"] = self.bc["dev"]
         ver.verify(self.state, self.conv, t["x"], t["dt"], t["B"], t["C"], self.A, self.D, self.cw, self.cb, z, y,
                    npv, k, layer=layer, **kw)
         torch.cuda.synchronize()
@@ -74,9 +81,15 @@ class Layer:
     def oracle_verify(self, batch, k, threads=None):
         s, p = self.s, self.np
         z = batch["z"] if s.flags & synth.FLAG_GATE else None
-        y, self.o_state, self.o_conv = oracle.verify(
-            self.o_state, self.o_conv, batch["x"], batch["dt"], batch["B"], batch["C"], p["A"], p["D"], p["cw"],
-            p["cb"], z, batch["n_prev"], k, s.flags & (synth.FLAG_GATE | synth.FLAG_CONV_SILU), threads=threads or oracle.host_threads())
+        core = s.flags & (synth.FLAG_GATE | synth.FLAG_CONV_SILU)
+        if self.bc:
+            y, self.o_state, self.o_conv, self.bc["o_window"] = oracle.verify_conv_bc(
+                self.o_state, self.o_conv, self.bc["o_window"], batch["x"], batch["dt"], batch["B"], batch["C"], p["A"], p["D"],
+                p["cw"], p["cb"], self.bc["taps"], self.bc["bias"], z, batch["n_prev"], k, core, threads=threads or oracle.host_threads())
+        else:
+            y, self.o_state, self.o_conv = oracle.verify(
+                self.o_state, self.o_conv, batch["x"], batch["dt"], batch["B"], batch["C"], p["A"], p["D"], p["cw"],
+                p["cb"], z, batch["n_prev"], k, core, threads=threads or oracle.host_threads())
         if self.norm:
             y = oracle.gated_rmsnorm(y, self.norm[0], self.norm[1])
         return y
@@ -90,6 +103,8 @@ class Layer:
         e_y = rel_l2(yg[valid], y_ref[valid])
         e_s = rel_l2(self.state.cpu().numpy(), self.o_state)
         e_c = np.abs(self.conv.float().cpu().numpy().astype(np.float64) - self.o_conv).max() if self.o_conv.size else 0.0
+        if self.bc:   # the window of the conv over B and C is a copy of input rows: exact
+            e_c = max(e_c, np.abs(self.bc["dev"][0].float().cpu().numpy().astype(np.float64) - self.bc["o_window"]).max())
         if y_gpu.dtype == torch.bfloat16:
             # y is a bf16 code: both sides take the rounding in the same precision.  Rounding the exact
             # output to bf16 costs 1.4e-3 .. 2.4e-3 relative L2 by itself on these workloads, so the

@@ -279,3 +279,32 @@ def test_gated_rmsnorm_of_the_output_rows(s, kernel, y_f32):
     assert ("stream" in name) == (kernel == STREAM)
     if tol:
         assert max(worst) <= tol
+
+
+# ------------------------------------------------------------------ conv over the B and C channels
+BC_FLAGS = synth.FLAG_GATE | synth.FLAG_CONV_SILU | synth.FLAG_CONV_BC
+BC_SHAPES = [
+    synth.Shape("bc_small_fp32", Bt=3, H=4, P=16, N=32, GB=2, GC=4, W=4, k=3, act="fp32", flags=BC_FLAGS),
+    synth.Shape("bc_bf16", Bt=2, H=8, P=64, N=128, GB=2, GC=8, W=4, k=4, act="bf16", flags=BC_FLAGS),
+    synth.Shape("bc_w3_norm", Bt=2, H=4, P=32, N=64, GB=1, GC=2, W=3, k=2, act="bf16", flags=BC_FLAGS | synth.FLAG_GATED_RMSNORM),
+]
+
+
+@pytest.mark.parametrize("s", BC_SHAPES, ids=lambda s: s.name)
+def test_conv_over_the_b_and_c_channels(s):
+    """MAMBA_SPEC_FLAG_CONV_BC: the B and C rows pass through their own rolling conv and activation before the
+    recurrence (oracle: verify_conv_bc); y in float32 so that the bound is 1e-5; the window of that conv is cached at
+    the verified position exactly.  Four rounds with replay, then a call without drafts."""
+    h = H()
+    worst, name = h.run_rounds(s, 4, kernel=0, first_j=2, y_f32=True, tol=1e-5, final_flush=True)
+    assert name == "generic"
+    assert max(worst) <= 1e-5
+
+
+def test_conv_over_b_and_c_is_refused_where_it_cannot_run():
+    from paper_2408_15237_b200 import binding
+    s = BC_SHAPES[1]
+    with pytest.raises(binding.MambaSpecError):      # the streaming kernel does not take it
+        H().make_verifier(s, STREAM)
+    with pytest.raises(binding.MambaSpecError):      # one window of B and C rows: no second snapshot
+        H().make_verifier(synth.replace(s, flags=s.flags | synth.FLAG_STATE_K), 0)
