@@ -184,10 +184,11 @@ def ver_n_prev(ver, batch):
     return binding.mamba_spec_get_n_prev(ver.ctx, batch)
 
 
-@pytest.mark.parametrize("s,kernel,selects", [(synth.CONFIGS[0], GENERIC, False), (synth.SWEEP[(4, 4)], STREAM, False),
-                                              (synth.SWEEP[(4, 4)], STREAM, True), (synth.SWEEP[(4, 4)], GENERIC, True),
-                                              (synth.CONFIGS[3], STREAM, True)])
-def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects):
+@pytest.mark.parametrize("s,kernel,selects,norm", [(synth.CONFIGS[0], GENERIC, False, False), (synth.SWEEP[(4, 4)], STREAM, False, False),
+                                              (synth.SWEEP[(4, 4)], STREAM, True, False), (synth.SWEEP[(4, 4)], GENERIC, True, False),
+                                              (synth.CONFIGS[3], STREAM, True, False), (synth.SWEEP[(4, 4)], STREAM, False, True),
+                                              (synth.SWEEP[(4, 4)], GENERIC, True, True)])
+def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects, norm):
     """The caller hands over only the k new rows per round (Sec. 4.2 "caching older entries"); the tokens accepted
     since the last call are replayed from the rows the library kept.  Two layers share the context (each has
     its own kept rows).  Mixed full and partial acceptance over eight rounds; returned rows, final caches and
@@ -196,6 +197,9 @@ def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects):
     from paper_2408_15237_b200 import binding
     n_layers = 2
     flags = s.flags | binding.FLAG_Y_F32 | ((binding.FLAG_STATE_K | binding.FLAG_COMMIT_SELECTS) if selects else 0)
+    flags |= binding.FLAG_GATED_RMSNORM if norm else 0      # (the normalising kernel then works on [batch][k] rows)
+    nw, neps = synth.norm_params(s, 0)
+    nkw = dict(norm_weight=h.dev(nw, torch.float32), norm_eps=neps) if norm else {}
     ver = binding.Verifier(s.Bt, s.H, s.P, s.N, s.GB, s.GC, s.W, s.k, act=s.act, flags=flags, kernel=kernel, n_layers=n_layers)
     ad = h.act_dtype(s)
     rounds = 8
@@ -219,7 +223,7 @@ def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects):
             y = torch.full((s.Bt, s.k, s.H, s.P), float("nan"), device="cuda", dtype=torch.float32)
             dA, dD, dcw, dcb = q["dev"]
             ver.verify_new(q["bufs"][0][0], q["bufs"][0][1], t["x"], t["dt"], t["B"], t["C"], dA, dD, dcw, dcb, t["z"], y, s.k,
-                           layer=l, state_k=q["bufs"][1][0] if selects else None, conv_state_k=q["bufs"][1][1] if selects else None)
+                           layer=l, state_k=q["bufs"][1][0] if selects else None, conv_state_k=q["bufs"][1][1] if selects else None, **nkw)
             torch.cuda.synchronize()
             assert ("stream" in ver.last_kernel) == (kernel == STREAM)
             yg = y.cpu().numpy().astype(np.float64)
@@ -234,7 +238,7 @@ def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects):
         dA, dD, dcw, dcb = q["dev"]
         y = torch.zeros((s.Bt, 1, s.H, s.P), device="cuda", dtype=torch.float32)
         ver.verify_new(q["bufs"][0][0], q["bufs"][0][1], None, None, None, None, dA, dD, dcw, dcb, None, y, 0, layer=l,
-                       state_k=q["bufs"][1][0] if selects else None, conv_state_k=q["bufs"][1][1] if selects else None)
+                       state_k=q["bufs"][1][0] if selects else None, conv_state_k=q["bufs"][1][1] if selects else None, **nkw)
     torch.cuda.synchronize()
     assert ver.status() == 0
     sel = ver.selection(s.Bt) if selects else [0] * s.Bt
@@ -243,6 +247,8 @@ def test_new_rows_only_with_the_library_side_row_store(s, kernel, selects):
         y_seq, st_seq, cv_seq = oracle.sequential(st, cv, q["stream"]["x"], q["stream"]["dt"], q["stream"]["B"], q["stream"]["C"],
                                                   A, D, cw, cb, q["stream"]["z"], cursor.astype(np.int32), s.flags,
                                                   threads=oracle.host_threads())
+        if norm:
+            y_seq = oracle.gated_rmsnorm(y_seq, nw, neps)
         for b in range(s.Bt):
             cur = q["bufs"][sel[b]]
             assert h.rel_l2(cur[0][b].cpu().numpy(), st_seq[b]) <= 1e-5, f"layer {l} sequence {b}: cache"
